@@ -1,0 +1,145 @@
+/* mop_moe.h -- C ABI of the B200 (sm_100a) routed-expert feed-forward layer.
+ *
+ * The layer is the MoE block of Section 2.1 of the paper ("Mixture-of-Experts" paragraph):
+ * E parallel expert networks and a router that sends each token to its top-k experts.
+ * Symbols follow Section 3.1: T tokens resident on the device (the paper's N), model width d
+ * (H), expert intermediate width f (I), E experts, routing degree k.  The buffers named Xp and
+ * H below are the O(N k H) and O(N_r I) terms of the activation peak in Eq. 4.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned, dense and
+ *     row-major with the shape given in the comment.  "bf16" means bfloat16 bit patterns.
+ *     The library allocates no tensor and keeps no pointer after the call's stream work ends.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     enqueue work and return; they do not synchronise.
+ *   - Argument errors are detected on the host before any launch and reported by the return
+ *     code; nothing is thrown, nothing aborts.  Kernels never trap: a wait that runs out of
+ *     its poll budget records a code in the context's status word, which mop_poll() reads.
+ *   - d and f must be multiples of 8 (16-byte rows); the tensor-core kernels further need
+ *     d and f to be multiples of 64 and otherwise the call uses the scalar kernels.
+ *   - No output is produced with atomics: results are bitwise reproducible run to run.
+ *   - A context is bound to one device and one shape; calls on one context must not overlap
+ *     on the GPU (they share its workspace).
+ */
+#ifndef MOP_MOE_H_
+#define MOP_MOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mop_ctx mop_ctx; /* opaque: shape, workspace, status word */
+
+typedef enum {
+    MOP_OK = 0,
+    MOP_ERR_INVALID_ARG = 1, /* null pointer, bad enum, k > E, ... */
+    MOP_ERR_SHAPE = 2,       /* sizes out of the supported range (T*k >= 2^31, E > 4096, ...) */
+    MOP_ERR_ALIGN = 3,       /* pointer not 16-byte aligned, or d / f not a multiple of 8 */
+    MOP_ERR_WORKSPACE = 4,   /* device allocation of the context's workspace failed */
+    MOP_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed */
+    MOP_ERR_UNSUPPORTED = 6, /* valid request that this build does not implement */
+    MOP_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (see mop_poll) */
+} mop_status;
+
+typedef enum { MOP_SCORE_SOFTMAX = 0, MOP_SCORE_SIGMOID = 1 } mop_score_fn;
+
+/* Where the per-expert router bias enters.  POST_SCORE: key = sigmoid(z) + b (selection
+ * only); PRE_LOGIT: key = z + b and the score is taken of z + b.  The bias never enters the
+ * gate numerator in POST_SCORE mode. */
+typedef enum { MOP_BIAS_NONE = 0, MOP_BIAS_POST_SCORE = 1, MOP_BIAS_PRE_LOGIT = 2 } mop_bias_mode;
+
+typedef enum { MOP_GEMM_AUTO = 0, MOP_GEMM_TENSOR = 1, MOP_GEMM_SCALAR = 2 } mop_gemm_path;
+
+typedef struct {
+    int32_t T, d, E, k, f;
+    int32_t score_fn;      /* mop_score_fn */
+    int32_t bias_mode;     /* mop_bias_mode; POST_SCORE requires MOP_SCORE_SIGMOID */
+    int32_t with_backward; /* 1: the context also holds the backward's intermediates */
+    int32_t dw_accumulate; /* 0: dW is overwritten (empty experts get zeros); 1: dW += */
+    int32_t gemm_path;     /* mop_gemm_path; AUTO = tensor cores when the shape allows */
+    int32_t host_io;       /* 1: the context also holds the activations of mop_moe_forward_host */
+} mop_moe_shape;
+
+/* Create / destroy a context on `device` (a CUDA ordinal).  mop_create allocates the
+ * workspace (mop_workspace_bytes) with cudaMalloc; every other call allocates nothing. */
+mop_status mop_create(mop_ctx** ctx, const mop_moe_shape* shape, int device);
+void mop_destroy(mop_ctx* ctx);
+size_t mop_workspace_bytes(const mop_moe_shape* shape);
+const char* mop_status_string(mop_status s);
+
+/* Synchronises `stream` and returns MOP_ERR_TIMEOUT if any kernel of this context recorded an
+ * exhausted wait since the last poll (then clears the word), MOP_ERR_CUDA on a CUDA error. */
+mop_status mop_poll(mop_ctx* ctx, void* stream);
+
+/* Number of kernels launched through this context since it was created. */
+int64_t mop_launch_count(const mop_ctx* ctx);
+
+/* Router (Section 2.1: "a lightweight router that sends each token to its top-k experts").
+ *   z[t,e]   = sum_i x[t,i] * W_r[i,e]: one fp32 fused multiply-add per i, i ascending.
+ *   key      = z | sigmoid(z) + bias | z + bias       (score_fn, bias_mode)
+ *   topk_idx = the k experts with the largest key, descending; equal keys -> lower id.
+ *   gate     = score of the selected expert / sum of the k selected scores.
+ * x [T,d] bf16; W_r [d,E] f32; bias [E] f32 (NULL iff MOP_BIAS_NONE);
+ * topk_idx [T,k] i32 out; topk_gate [T,k] f32 out; logits_opt [T,E] f32 out or NULL. */
+mop_status mop_moe_route(mop_ctx* ctx, const void* x, const float* W_r, const float* bias, int32_t* topk_idx,
+                         float* topk_gate, float* logits_opt, void* stream);
+
+/* Count and prefix-sum permutation of assignments a = t*k + j into expert-contiguous rows
+ * (the buffer of N k rows of width H in Eq. 4).
+ *   counts[e]   = number of assignments to expert e;   offsets = exclusive scan, offsets[E] = T*k
+ *   perm_row[a] = offsets[idx[a]] + (number of a' < a with the same expert)     (stable)
+ *   row_src     = inverse of perm_row;   Xp[p,:] = x[row_src[p] / k, :]
+ * x [T,d] bf16; topk_idx [T,k]; counts [E]; offsets [E+1]; perm_row, row_src [T*k] i32 out;
+ * Xp [T*k,d] bf16 out.  Indices outside [0,E) are a caller error (rows are dropped). */
+mop_status mop_moe_permute(mop_ctx* ctx, const void* x, const int32_t* topk_idx, int32_t* counts, int32_t* offsets,
+                           int32_t* perm_row, int32_t* row_src, void* Xp, void* stream);
+
+/* Grouped SwiGLU expert feed-forward over the permuted rows (Section 2.1 "expert networks";
+ * H is the N_r I term of Eq. 4).  For the rows p of expert e (offsets[e] <= p < offsets[e+1]):
+ *   G = Xp W_gate[e], U = Xp W_up[e] (fp32 accumulation);  H = bf16(silu(G) * U)
+ *   Yp[p,:] = bf16( gate(p) * (H[p,:] W_down[e]) ),  gate(p) = topk_gate[row_src[p]]
+ * Xp [T*k,d] bf16; offsets [E+1]; row_src [T*k]; topk_gate [T,k] f32;
+ * W_gate, W_up [E,d,f] bf16; W_down [E,f,d] bf16;
+ * G_save, U_save [T*k,f] bf16 out, both NULL (forward only) or both set (kept for backward);
+ * H [T*k,f] bf16 out (required); Yp [T*k,d] bf16 out. */
+mop_status mop_moe_expert_ffn_fwd(mop_ctx* ctx, const void* Xp, const int32_t* offsets, const int32_t* row_src,
+                                  const float* topk_gate, const void* W_gate, const void* W_up, const void* W_down,
+                                  void* G_save, void* U_save, void* H, void* Yp, void* stream);
+
+/* Unpermute-combine: Y[t,:] = bf16( sum_j Yp[perm_row[t*k+j], :] ), fp32 sum, j ascending.
+ * (The gate was applied by mop_moe_expert_ffn_fwd.)  Also used for dX from dXp.
+ * Yp [T*k,d] bf16; perm_row [T*k]; Y [T,d] bf16 out. */
+mop_status mop_moe_combine(mop_ctx* ctx, const void* Yp, const int32_t* perm_row, void* Y, void* stream);
+
+/* Backward of expert_ffn_fwd followed by combine, with topk_idx and topk_gate as inputs of
+ * the function (the router's own backward is outside this library).  With p <-> (t,j,e):
+ *   dgate[t,j] = < dY[t,:] W_down[e]^T , H[p,:] >
+ *   dH = gate * dY[t,:] W_down[e]^T;  dG = dH * U * s(G) (1 + G (1 - s(G)));  dU = dH * silu(G)
+ *   dX[t,:]    = sum_j ( dG[p_j,:] W_gate[e_j]^T + dU[p_j,:] W_up[e_j]^T )
+ *   dW_gate[e] = Xp_e^T dG_e;  dW_up[e] = Xp_e^T dU_e;  dW_down[e] = (gate * H_e)^T dY_e
+ * dY [T,d] bf16; Xp, G_save, U_save, H, offsets, perm_row, row_src, topk_gate, W_* as above;
+ * dX [T,d] bf16 out; dW_gate, dW_up [E,d,f] f32 out; dW_down [E,f,d] f32 out;
+ * dgate [T,k] f32 out.  Needs a context created with with_backward = 1. */
+mop_status mop_moe_expert_ffn_bwd(mop_ctx* ctx, const void* dY, const void* Xp, const void* G_save,
+                                  const void* U_save, const void* H, const int32_t* offsets, const int32_t* perm_row,
+                                  const int32_t* row_src, const float* topk_gate, const void* W_gate,
+                                  const void* W_up, const void* W_down, void* dX, float* dW_gate, float* dW_up,
+                                  float* dW_down, float* dgate, void* stream);
+
+/* Whole forward with HOST buffers (pageable or pinned): copies x in, runs route, permute,
+ * expert_ffn_fwd and combine on `stream`, copies Y, topk_idx and topk_gate back, and
+ * synchronises.  Weights stay on the device (they are parameters, not step inputs).
+ * Scratch activations come from the context (created with this shape).
+ * x_host [T,d] bf16; Y_host [T,d] bf16 out; idx_host [T,k] i32 out or NULL;
+ * gate_host [T,k] f32 out or NULL. */
+mop_status mop_moe_forward_host(mop_ctx* ctx, const void* x_host, const float* W_r, const float* bias,
+                                const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
+                                int32_t* idx_host, float* gate_host, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOP_MOE_H_ */

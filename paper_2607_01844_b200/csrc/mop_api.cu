@@ -1,0 +1,455 @@
+// C ABI of the routed-expert layer: argument checks, workspace, launches.  See include/mop_moe.h
+// for the contract of every entry point.
+#include "../../include/mop_moe.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <new>
+
+#include "common.cuh"
+#include "epilogue.cuh"
+#include "gemm_scalar.cuh"
+#include "gemm_tc.cuh"
+#include "permute.cuh"
+#include "route.cuh"
+
+using namespace mop;
+
+struct mop_ctx {
+    mop_moe_shape s;
+    int device;
+    int sm_count;
+    int64_t launches;
+    bool tensor_ok;      // shape admits the tensor-core kernels
+    // workspace (one allocation)
+    char* ws;
+    size_t ws_bytes;
+    float* z;            // [T,E] logits
+    int32_t* partial;    // [units,E] histogram partials -> unit bases
+    int32_t* tiles;      // tile tables of the grouped GEMMs
+    int32_t* status;     // device status word
+    float* part;         // [ntile_max, M] partial dot products for dgate
+    bf16 *dYp, *dG, *dU, *gH, *dXp;  // backward intermediates
+    // host-buffer entry point scratch
+    bf16 *hx, *hXp, *hH, *hYp, *hY;
+    int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
+    float* hgate;
+    TcPlan plan;
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp;
+    size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
+    size_t total;
+};
+
+int perm_units(const mop_moe_shape& s) { return ceil_div(s.T * s.k, PERM_SEG); }
+int part_tiles(const mop_moe_shape& s) { return ceil_div(s.f, 64); }
+
+Layout make_layout(const mop_moe_shape& s) {
+    Layout L{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o += align_up(bytes); return r; };
+    const size_t T = s.T, d = s.d, E = s.E, k = s.k, f = s.f, M = T * k;
+    L.z = take(T * E * 4);
+    L.partial = take((size_t)perm_units(s) * E * 4 + 4);
+    L.tiles = take(tc_tile_table_bytes(s.T * s.k, s.E));
+    L.status = take(256);
+    if (s.with_backward) {
+        L.part = take((size_t)part_tiles(s) * M * 4);
+        L.dYp = take(M * d * 2);
+        L.dG = take(M * f * 2);
+        L.dU = take(M * f * 2);
+        L.gH = take(M * f * 2);
+        L.dXp = take(M * d * 2);
+    }
+    if (s.host_io) {
+        L.hx = take(T * d * 2);
+        L.hXp = take(M * d * 2);
+        L.hH = take(M * f * 2);
+        L.hYp = take(M * d * 2);
+        L.hY = take(T * d * 2);
+        L.hidx = take(M * 4);
+        L.hcounts = take(E * 4);
+        L.hoffsets = take((E + 1) * 4);
+        L.hperm = take(M * 4);
+        L.hsrc = take(M * 4);
+        L.hgate = take(M * 4);
+    }
+    L.total = o;
+    return L;
+}
+
+mop_status check_shape(const mop_moe_shape* s) {
+    if (!s) return MOP_ERR_INVALID_ARG;
+    if (s->T < 0 || s->d < 1 || s->E < 1 || s->k < 1 || s->f < 1) return MOP_ERR_INVALID_ARG;
+    if (s->k > s->E) return MOP_ERR_INVALID_ARG;
+    if (s->score_fn != MOP_SCORE_SOFTMAX && s->score_fn != MOP_SCORE_SIGMOID) return MOP_ERR_INVALID_ARG;
+    if (s->bias_mode < MOP_BIAS_NONE || s->bias_mode > MOP_BIAS_PRE_LOGIT) return MOP_ERR_INVALID_ARG;
+    if (s->bias_mode == MOP_BIAS_POST_SCORE && s->score_fn != MOP_SCORE_SIGMOID) return MOP_ERR_INVALID_ARG;
+    if (s->gemm_path < MOP_GEMM_AUTO || s->gemm_path > MOP_GEMM_SCALAR) return MOP_ERR_INVALID_ARG;
+    if ((long long)s->T * s->k >= (1ll << 31) - 4096) return MOP_ERR_SHAPE;
+    if (s->E > SEL_MAX_E || s->k > 32) return MOP_ERR_SHAPE;
+    if ((long long)s->T * s->d >= (1ll << 40) || (long long)s->d * s->f >= (1ll << 31)) return MOP_ERR_SHAPE;
+    if (s->d % 8 || s->f % 8) return MOP_ERR_ALIGN;
+    return MOP_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+#define REQ_PTR(p)                                      \
+    do {                                                \
+        if (!(p)) return MOP_ERR_INVALID_ARG;           \
+        if (!aligned16(p)) return MOP_ERR_ALIGN;        \
+    } while (0)
+
+#define CUDA_OK(expr)                                   \
+    do {                                                \
+        if ((expr) != cudaSuccess) return MOP_ERR_CUDA; \
+    } while (0)
+
+inline mop_status after_launch(mop_ctx* c, int n = 1) {
+    c->launches += n;
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess && (prev == dev || cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        int cur;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+bool use_tensor(const mop_ctx* c) { return c->tensor_ok && c->s.gemm_path != MOP_GEMM_SCALAR; }
+
+// ---- scalar-path launches ---------------------------------------------------------------
+mop_status launch_scalar(mop_ctx* c, const ScalarGemmArgs& g, cudaStream_t st) {
+    dim3 grid(ceil_div(g.N, SG_BN), c->s.E);
+    scalar_grouped_gemm_kernel<<<grid, 256, 0, st>>>(g);
+    return after_launch(c);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* mop_status_string(mop_status s) {
+    switch (s) {
+        case MOP_OK: return "ok";
+        case MOP_ERR_INVALID_ARG: return "invalid argument";
+        case MOP_ERR_SHAPE: return "shape out of supported range";
+        case MOP_ERR_ALIGN: return "misaligned pointer or row size";
+        case MOP_ERR_WORKSPACE: return "workspace allocation failed";
+        case MOP_ERR_CUDA: return "CUDA call failed";
+        case MOP_ERR_UNSUPPORTED: return "unsupported request";
+        case MOP_ERR_TIMEOUT: return "device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+size_t mop_workspace_bytes(const mop_moe_shape* shape) {
+    if (check_shape(shape) != MOP_OK) return 0;
+    return make_layout(*shape).total;
+}
+
+mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
+    if (!out) return MOP_ERR_INVALID_ARG;
+    *out = nullptr;
+    mop_status st = check_shape(shape);
+    if (st != MOP_OK) return st;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) return MOP_ERR_CUDA;
+    if (device < 0 || device >= ndev) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    mop_ctx* c = new (std::nothrow) mop_ctx();
+    if (!c) return MOP_ERR_WORKSPACE;
+    c->s = *shape;
+    c->device = device;
+    c->launches = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return MOP_ERR_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    c->tensor_ok = (prop.major == 10) && tc_shape_supported(shape->d, shape->f);
+    if (shape->gemm_path == MOP_GEMM_TENSOR && !c->tensor_ok) { delete c; return MOP_ERR_UNSUPPORTED; }
+    const Layout L = make_layout(*shape);
+    c->ws_bytes = L.total;
+    if (cudaMalloc(&c->ws, L.total) != cudaSuccess) { cudaGetLastError(); delete c; return MOP_ERR_WORKSPACE; }
+    char* w = c->ws;
+    c->z = reinterpret_cast<float*>(w + L.z);
+    c->partial = reinterpret_cast<int32_t*>(w + L.partial);
+    c->tiles = reinterpret_cast<int32_t*>(w + L.tiles);
+    c->status = reinterpret_cast<int32_t*>(w + L.status);
+    if (shape->with_backward) {
+        c->part = reinterpret_cast<float*>(w + L.part);
+        c->dYp = reinterpret_cast<bf16*>(w + L.dYp);
+        c->dG = reinterpret_cast<bf16*>(w + L.dG);
+        c->dU = reinterpret_cast<bf16*>(w + L.dU);
+        c->gH = reinterpret_cast<bf16*>(w + L.gH);
+        c->dXp = reinterpret_cast<bf16*>(w + L.dXp);
+    }
+    if (shape->host_io) {
+        c->hx = reinterpret_cast<bf16*>(w + L.hx);
+        c->hXp = reinterpret_cast<bf16*>(w + L.hXp);
+        c->hH = reinterpret_cast<bf16*>(w + L.hH);
+        c->hYp = reinterpret_cast<bf16*>(w + L.hYp);
+        c->hY = reinterpret_cast<bf16*>(w + L.hY);
+        c->hidx = reinterpret_cast<int32_t*>(w + L.hidx);
+        c->hcounts = reinterpret_cast<int32_t*>(w + L.hcounts);
+        c->hoffsets = reinterpret_cast<int32_t*>(w + L.hoffsets);
+        c->hperm = reinterpret_cast<int32_t*>(w + L.hperm);
+        c->hsrc = reinterpret_cast<int32_t*>(w + L.hsrc);
+        c->hgate = reinterpret_cast<float*>(w + L.hgate);
+    }
+    if (cudaMemset(c->status, 0, 256) != cudaSuccess) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
+    if (c->tensor_ok) {
+        st = tc_plan_init(&c->plan, *shape, c->sm_count);
+        if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
+    }
+    *out = c;
+    return MOP_OK;
+}
+
+void mop_destroy(mop_ctx* c) {
+    if (!c) return;
+    DeviceGuard guard(c->device);
+    cudaFree(c->ws);
+    delete c;
+}
+
+int64_t mop_launch_count(const mop_ctx* c) { return c ? c->launches : 0; }
+
+mop_status mop_poll(mop_ctx* c, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    CUDA_OK(cudaMemcpyAsync(&word, c->status, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    if (word != 0) {
+        CUDA_OK(cudaMemsetAsync(c->status, 0, 4, st));
+        CUDA_OK(cudaStreamSynchronize(st));
+        return MOP_ERR_TIMEOUT;
+    }
+    return MOP_OK;
+}
+
+mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const float* bias, int32_t* topk_idx,
+                         float* topk_gate, float* logits_opt, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    REQ_PTR(x); REQ_PTR(W_r); REQ_PTR(topk_idx); REQ_PTR(topk_gate);
+    if ((c->s.bias_mode != MOP_BIAS_NONE) != (bias != nullptr)) return MOP_ERR_INVALID_ARG;
+    if (logits_opt && !aligned16(logits_opt)) return MOP_ERR_ALIGN;
+    const mop_moe_shape& s = c->s;
+    if (s.T == 0) return MOP_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* z = logits_opt ? logits_opt : c->z;
+    dim3 grid(ceil_div(s.T, SC_TT), ceil_div(s.E, SC_TE));
+    route_score_kernel<<<grid, 256, 0, st>>>(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E);
+    mop_status r = after_launch(c);
+    if (r != MOP_OK) return r;
+    const size_t smem = (size_t)SEL_WARPS * 2 * s.E * sizeof(float);
+    route_select_kernel<<<ceil_div(s.T, SEL_WARPS), SEL_WARPS * 32, smem, st>>>(z, bias, topk_idx, topk_gate, s.T, s.E,
+                                                                               s.k, s.score_fn, s.bias_mode);
+    return after_launch(c);
+}
+
+mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, int32_t* counts, int32_t* offsets,
+                           int32_t* perm_row, int32_t* row_src, void* Xp, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    REQ_PTR(x); REQ_PTR(topk_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR(perm_row); REQ_PTR(row_src); REQ_PTR(Xp);
+    const mop_moe_shape& s = c->s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int M = s.T * s.k;
+    const int units = perm_units(s);
+    const size_t smem = (size_t)PERM_WARPS * s.E * sizeof(int32_t);
+    mop_status r;
+    if (units > 0) {
+        perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, M, s.E);
+        if ((r = after_launch(c)) != MOP_OK) return r;
+    }
+    perm_scan_kernel<<<1, 1024, (s.E + 1) * sizeof(int32_t), st>>>(c->partial, counts, offsets, units, s.E);
+    if ((r = after_launch(c)) != MOP_OK) return r;
+    if (units == 0) return MOP_OK;
+    perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, perm_row,
+                                                                                row_src, M, s.E);
+    if ((r = after_launch(c)) != MOP_OK) return r;
+    const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
+    scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, s.T,
+                                                s.k, s.d / 8);
+    return after_launch(c);
+}
+
+mop_status mop_moe_combine(mop_ctx* c, const void* Yp, const int32_t* perm_row, void* Y, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    REQ_PTR(Yp); REQ_PTR(perm_row); REQ_PTR(Y);
+    const mop_moe_shape& s = c->s;
+    if (s.T == 0) return MOP_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
+    combine_rows_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(Yp), perm_row, static_cast<uint4*>(Y), s.T, s.k, s.d / 8);
+    return after_launch(c);
+}
+
+mop_status mop_moe_expert_ffn_fwd(mop_ctx* c, const void* Xp, const int32_t* offsets, const int32_t* row_src,
+                                  const float* topk_gate, const void* W_gate, const void* W_up, const void* W_down,
+                                  void* G_save, void* U_save, void* H, void* Yp, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    REQ_PTR(Xp); REQ_PTR(offsets); REQ_PTR(row_src); REQ_PTR(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up);
+    REQ_PTR(W_down); REQ_PTR(H); REQ_PTR(Yp);
+    if ((G_save == nullptr) != (U_save == nullptr)) return MOP_ERR_INVALID_ARG;
+    if (G_save && (!aligned16(G_save) || !aligned16(U_save))) return MOP_ERR_ALIGN;
+    const mop_moe_shape& s = c->s;
+    if (s.T == 0) return MOP_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int M = s.T * s.k;
+    if (use_tensor(c)) {
+        TcFwdArgs a{};
+        a.Xp = static_cast<const bf16*>(Xp); a.offsets = offsets; a.row_src = row_src; a.gate = topk_gate;
+        a.W_gate = static_cast<const bf16*>(W_gate); a.W_up = static_cast<const bf16*>(W_up);
+        a.W_down = static_cast<const bf16*>(W_down);
+        a.G_save = static_cast<bf16*>(G_save); a.U_save = static_cast<bf16*>(U_save);
+        a.H = static_cast<bf16*>(H); a.Yp = static_cast<bf16*>(Yp);
+        int n = 0;
+        mop_status r = tc_ffn_fwd(&c->plan, a, c->tiles, c->status, st, &n);
+        c->launches += n;
+        return r;
+    }
+    ScalarGemmArgs g{};
+    g.A[0] = g.A[1] = static_cast<const bf16*>(Xp);
+    g.B[0] = static_cast<const bf16*>(W_gate); g.B[1] = static_cast<const bf16*>(W_up);
+    g.sAm = s.d; g.sAk = 1; g.sBk = s.f; g.sBn = 1; g.sBe = (long)s.d * s.f;
+    g.offsets = offsets; g.ragged_k = 0; g.N = s.f; g.Kfix = s.d; g.npairs = 2; g.dual_acc = 1; g.epi = EPI_SWIGLU;
+    g.ep.out0 = static_cast<bf16*>(H); g.ep.out1 = static_cast<bf16*>(G_save); g.ep.out2 = static_cast<bf16*>(U_save);
+    g.ep.ldo = s.f; g.ep.M_total = M;
+    mop_status r = launch_scalar(c, g, st);
+    if (r != MOP_OK) return r;
+    ScalarGemmArgs h{};
+    h.A[0] = static_cast<const bf16*>(H); h.B[0] = static_cast<const bf16*>(W_down);
+    h.sAm = s.f; h.sAk = 1; h.sBk = s.d; h.sBn = 1; h.sBe = (long)s.d * s.f;
+    h.offsets = offsets; h.ragged_k = 0; h.N = s.d; h.Kfix = s.f; h.npairs = 1; h.epi = EPI_GATE;
+    h.ep.out0 = static_cast<bf16*>(Yp); h.ep.gate = topk_gate; h.ep.row_src = row_src; h.ep.ldo = s.d; h.ep.M_total = M;
+    return launch_scalar(c, h, st);
+}
+
+mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, const void* G_save,
+                                  const void* U_save, const void* H, const int32_t* offsets, const int32_t* perm_row,
+                                  const int32_t* row_src, const float* topk_gate, const void* W_gate,
+                                  const void* W_up, const void* W_down, void* dX, float* dW_gate, float* dW_up,
+                                  float* dW_down, float* dgate, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (!c->s.with_backward) return MOP_ERR_UNSUPPORTED;
+    REQ_PTR(dY); REQ_PTR(Xp); REQ_PTR(G_save); REQ_PTR(U_save); REQ_PTR(H); REQ_PTR(offsets); REQ_PTR(perm_row);
+    REQ_PTR(row_src); REQ_PTR(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up); REQ_PTR(W_down); REQ_PTR(dX);
+    REQ_PTR(dW_gate); REQ_PTR(dW_up); REQ_PTR(dW_down); REQ_PTR(dgate);
+    const mop_moe_shape& s = c->s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int M = s.T * s.k;
+    mop_status r;
+    if (s.T > 0) {
+        // dYp[p,:] = dY[t,:]  (unscaled; the gate enters through dH and gate*H)
+        const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
+        scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dY), reinterpret_cast<uint4*>(c->dYp),
+                                                    perm_row, s.T, s.k, s.d / 8);
+        if ((r = after_launch(c)) != MOP_OK) return r;
+    }
+    int ntile_part = 0;
+    if (use_tensor(c)) {
+        TcBwdArgs a{};
+        a.dYp = c->dYp; a.Xp = static_cast<const bf16*>(Xp); a.G_save = static_cast<const bf16*>(G_save);
+        a.U_save = static_cast<const bf16*>(U_save); a.H = static_cast<const bf16*>(H);
+        a.offsets = offsets; a.row_src = row_src; a.gate = topk_gate;
+        a.W_gate = static_cast<const bf16*>(W_gate); a.W_up = static_cast<const bf16*>(W_up);
+        a.W_down = static_cast<const bf16*>(W_down);
+        a.dG = c->dG; a.dU = c->dU; a.gH = c->gH; a.dXp = c->dXp; a.part = c->part;
+        a.dW_gate = dW_gate; a.dW_up = dW_up; a.dW_down = dW_down; a.accumulate = s.dw_accumulate;
+        int n = 0;
+        r = tc_ffn_bwd(&c->plan, a, c->tiles, c->status, st, &n, &ntile_part);
+        c->launches += n;
+        if (r != MOP_OK) return r;
+    } else {
+        if (s.T > 0) {
+            ScalarGemmArgs g{};  // dHu = dYp W_down^T, SwiGLU backward in the epilogue
+            g.A[0] = c->dYp; g.B[0] = static_cast<const bf16*>(W_down);
+            g.sAm = s.d; g.sAk = 1; g.sBk = 1; g.sBn = s.d; g.sBe = (long)s.d * s.f;
+            g.offsets = offsets; g.N = s.f; g.Kfix = s.d; g.npairs = 1; g.epi = EPI_DH;
+            g.ep.out0 = c->dG; g.ep.out1 = c->dU; g.ep.out2 = c->gH;
+            g.ep.in0 = static_cast<const bf16*>(G_save); g.ep.in1 = static_cast<const bf16*>(U_save);
+            g.ep.in2 = static_cast<const bf16*>(H);
+            g.ep.gate = topk_gate; g.ep.row_src = row_src; g.ep.part = c->part; g.ep.ldo = s.f; g.ep.M_total = M;
+            if ((r = launch_scalar(c, g, st)) != MOP_OK) return r;
+            ntile_part = ceil_div(s.f, SG_BN);
+            ScalarGemmArgs h{};  // dXp = dG W_gate^T + dU W_up^T
+            h.A[0] = c->dG; h.A[1] = c->dU;
+            h.B[0] = static_cast<const bf16*>(W_gate); h.B[1] = static_cast<const bf16*>(W_up);
+            h.sAm = s.f; h.sAk = 1; h.sBk = 1; h.sBn = s.f; h.sBe = (long)s.d * s.f;
+            h.offsets = offsets; h.N = s.d; h.Kfix = s.f; h.npairs = 2; h.dual_acc = 0; h.epi = EPI_BF16;
+            h.ep.out0 = c->dXp; h.ep.ldo = s.d; h.ep.M_total = M;
+            if ((r = launch_scalar(c, h, st)) != MOP_OK) return r;
+        }
+        // weight gradients (ragged K = the expert's rows); run even for T = 0 so that dW is defined
+        ScalarGemmArgs w{};
+        w.offsets = offsets; w.ragged_k = 1; w.npairs = 1; w.epi = EPI_F32; w.ep.accumulate = s.dw_accumulate;
+        w.A[0] = c->gH; w.sAm = 1; w.sAk = s.f; w.B[0] = c->dYp; w.sBk = s.d; w.sBn = 1;
+        w.Mfix = s.f; w.N = s.d; w.ep.outf = dW_down;
+        if ((r = launch_scalar(c, w, st)) != MOP_OK) return r;
+        w.A[0] = static_cast<const bf16*>(Xp); w.sAm = 1; w.sAk = s.d; w.B[0] = c->dG; w.sBk = s.f; w.sBn = 1;
+        w.Mfix = s.d; w.N = s.f; w.ep.outf = dW_gate;
+        if ((r = launch_scalar(c, w, st)) != MOP_OK) return r;
+        w.B[0] = c->dU; w.ep.outf = dW_up;
+        if ((r = launch_scalar(c, w, st)) != MOP_OK) return r;
+    }
+    if (s.T == 0) return MOP_OK;
+    dgate_reduce_kernel<<<ceil_div(M, 256), 256, 0, st>>>(c->part, perm_row, dgate, M, ntile_part);
+    if ((r = after_launch(c)) != MOP_OK) return r;
+    return mop_moe_combine(c, c->dXp, perm_row, dX, stream);
+}
+
+mop_status mop_moe_forward_host(mop_ctx* c, const void* x_host, const float* W_r, const float* bias,
+                                const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
+                                int32_t* idx_host, float* gate_host, void* stream) {
+    if (!c || !x_host || !Y_host) return MOP_ERR_INVALID_ARG;
+    if (!c->s.host_io) return MOP_ERR_UNSUPPORTED;
+    const mop_moe_shape& s = c->s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t M = (size_t)s.T * s.k;
+    CUDA_OK(cudaMemcpyAsync(c->hx, x_host, (size_t)s.T * s.d * 2, cudaMemcpyHostToDevice, st));
+    mop_status r;
+    if ((r = mop_moe_route(c, c->hx, W_r, bias, c->hidx, c->hgate, nullptr, stream)) != MOP_OK) return r;
+    if ((r = mop_moe_permute(c, c->hx, c->hidx, c->hcounts, c->hoffsets, c->hperm, c->hsrc, c->hXp, stream)) != MOP_OK)
+        return r;
+    if ((r = mop_moe_expert_ffn_fwd(c, c->hXp, c->hoffsets, c->hsrc, c->hgate, W_gate, W_up, W_down, nullptr, nullptr,
+                                    c->hH, c->hYp, stream)) != MOP_OK)
+        return r;
+    if ((r = mop_moe_combine(c, c->hYp, c->hperm, c->hY, stream)) != MOP_OK) return r;
+    CUDA_OK(cudaMemcpyAsync(Y_host, c->hY, (size_t)s.T * s.d * 2, cudaMemcpyDeviceToHost, st));
+    if (idx_host) CUDA_OK(cudaMemcpyAsync(idx_host, c->hidx, M * 4, cudaMemcpyDeviceToHost, st));
+    if (gate_host) CUDA_OK(cudaMemcpyAsync(gate_host, c->hgate, M * 4, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    return MOP_OK;
+}
+
+}  // extern "C"

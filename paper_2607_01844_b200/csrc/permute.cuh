@@ -1,0 +1,199 @@
+// Count / prefix-sum permutation of token-expert assignments into expert-contiguous rows, and the
+// row movers (scatter x -> Xp, k-row combine Yp -> Y).  No atomics anywhere: the order inside an
+// expert is the assignment id, fixed by a two-level (warp segment, expert) prefix sum.
+#pragma once
+#include "common.cuh"
+
+namespace mop {
+
+constexpr int PERM_SEG = 512;    // assignments walked by one warp ("unit")
+constexpr int PERM_WARPS = 4;    // warps per block in the histogram / rank kernels
+
+// Histogram per unit: partial[u][e] = number of assignments of unit u that go to expert e.
+__global__ void __launch_bounds__(PERM_WARPS * 32) perm_hist_kernel(const int32_t* __restrict__ idx,
+                                                                    int32_t* __restrict__ partial, int M, int E) {
+    extern __shared__ int32_t perm_smem[];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    int32_t* cnt = perm_smem + (size_t)warp * E;
+    const int unit = blockIdx.x * PERM_WARPS + warp;
+    const int a0 = unit * PERM_SEG;
+    if (a0 >= M) return;
+    for (int e = lane; e < E; e += 32) cnt[e] = 0;
+    __syncwarp();
+    for (int it = 0; it < PERM_SEG / 32; ++it) {
+        const int a = a0 + it * 32 + lane;
+        int e = (a < M) ? idx[a] : -1;
+        if (e < 0 || e >= E) e = -1;
+        const uint32_t same = __match_any_sync(0xffffffffu, e);
+        if (e >= 0 && lane == __ffs(same) - 1) cnt[e] += __popc(same);
+        __syncwarp();
+    }
+    for (int e = lane; e < E; e += 32) partial[(size_t)unit * E + e] = cnt[e];
+}
+
+// Scan: counts, offsets (exclusive scan over experts) and, in place of partial[u][e], the first
+// row of unit u inside expert e.  One block; thread e owns expert e (strided if E > blockDim).
+__global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ partial, int32_t* __restrict__ counts,
+                                                         int32_t* __restrict__ offsets, int units, int E) {
+    extern __shared__ int32_t scan_smem[];  // E + 1
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int32_t run = 0;
+        for (int u = 0; u < units; ++u) {
+            const int32_t c = partial[(size_t)u * E + e];
+            partial[(size_t)u * E + e] = run;
+            run += c;
+        }
+        counts[e] = run;
+        scan_smem[e] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        // exclusive scan over E by one warp, 32 experts per step
+        int32_t carry = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + threadIdx.x;
+            const int32_t c = (e < E) ? scan_smem[e] : 0;
+            int32_t inc = c;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t o = __shfl_up_sync(0xffffffffu, inc, off);
+                if ((int)threadIdx.x >= off) inc += o;
+            }
+            if (e < E) scan_smem[e] = carry + inc - c;
+            carry += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (threadIdx.x == 0) scan_smem[E] = carry;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) offsets[e] = scan_smem[e];
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        const int32_t o = scan_smem[e];
+        for (int u = 0; u < units; ++u) partial[(size_t)u * E + e] += o;
+    }
+}
+
+// Rank: second walk over the same segments; perm_row[a] = base[u][e] + rank inside the unit.
+__global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_t* __restrict__ idx,
+                                                                    const int32_t* __restrict__ base,
+                                                                    int32_t* __restrict__ perm_row,
+                                                                    int32_t* __restrict__ row_src, int M, int E) {
+    extern __shared__ int32_t perm_smem[];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    int32_t* run = perm_smem + (size_t)warp * E;
+    const int unit = blockIdx.x * PERM_WARPS + warp;
+    const int a0 = unit * PERM_SEG;
+    if (a0 >= M) return;
+    for (int e = lane; e < E; e += 32) run[e] = base[(size_t)unit * E + e];
+    __syncwarp();
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int it = 0; it < PERM_SEG / 32; ++it) {
+        const int a = a0 + it * 32 + lane;
+        int e = (a < M) ? idx[a] : -1;
+        if (e < 0 || e >= E) e = -1;
+        const uint32_t same = __match_any_sync(0xffffffffu, e);
+        int32_t p = -1;
+        if (e >= 0) p = run[e] + __popc(same & lt);
+        __syncwarp();
+        if (e >= 0 && lane == __ffs(same) - 1) run[e] += __popc(same);
+        __syncwarp();
+        if (a < M) {
+            perm_row[a] = p;
+            if (p >= 0) row_src[p] = a;
+        }
+    }
+}
+
+// Scatter rows: one warp per token reads x[t,:] once (16-byte vectors, coalesced) and writes it to
+// its k destination rows.  Used for x -> Xp and for dY -> dYp.
+__global__ void __launch_bounds__(256) scatter_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
+                                                           const int32_t* __restrict__ perm_row, int T, int k,
+                                                           int vec_per_row) {
+    const int warps_per_block = blockDim.x / 32;
+    const int lane = threadIdx.x % 32;
+    for (int t = blockIdx.x * warps_per_block + threadIdx.x / 32; t < T; t += gridDim.x * warps_per_block) {
+        int32_t myrow = -1;
+        if (lane < k) myrow = perm_row[(size_t)t * k + lane];  // k <= 32 checked on the host
+        const uint4* s = src + (size_t)t * vec_per_row;
+        for (int c0 = 0; c0 < vec_per_row; c0 += 128) {
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int c = c0 + q * 32 + lane;
+                if (c < vec_per_row) v[q] = __ldg(s + c);
+            }
+            for (int j = 0; j < k; ++j) {
+                const int32_t p = __shfl_sync(0xffffffffu, myrow, j);
+                if (p < 0) continue;
+                uint4* o = dst + (size_t)p * vec_per_row;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int c = c0 + q * 32 + lane;
+                    if (c < vec_per_row) __stcs(o + c, v[q]);
+                }
+            }
+        }
+    }
+}
+
+// Combine: Y[t,:] = bf16(sum_j Yp[perm_row[t*k+j],:]) with the k-row sum kept in fp32 registers,
+// j ascending.  One warp per token, 16-byte vectors.
+__global__ void __launch_bounds__(256) combine_rows_kernel(const uint4* __restrict__ Yp,
+                                                           const int32_t* __restrict__ perm_row,
+                                                           uint4* __restrict__ Y, int T, int k, int vec_per_row) {
+    const int warps_per_block = blockDim.x / 32;
+    const int lane = threadIdx.x % 32;
+    for (int t = blockIdx.x * warps_per_block + threadIdx.x / 32; t < T; t += gridDim.x * warps_per_block) {
+        int32_t myrow = -1;
+        if (lane < k) myrow = perm_row[(size_t)t * k + lane];
+        for (int c0 = 0; c0 < vec_per_row; c0 += 64) {
+            float acc[2][8];
+#pragma unroll
+            for (int q = 0; q < 2; ++q)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[q][i] = 0.0f;
+            for (int j = 0; j < k; ++j) {
+                const int32_t p = __shfl_sync(0xffffffffu, myrow, j);
+                if (p < 0) continue;
+                const uint4* r = Yp + (size_t)p * vec_per_row;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int c = c0 + q * 32 + lane;
+                    if (c < vec_per_row) {
+                        const uint4 v = __ldcs(r + c);
+                        acc[q][0] += bf16_lo(v.x); acc[q][1] += bf16_hi(v.x);
+                        acc[q][2] += bf16_lo(v.y); acc[q][3] += bf16_hi(v.y);
+                        acc[q][4] += bf16_lo(v.z); acc[q][5] += bf16_hi(v.z);
+                        acc[q][6] += bf16_lo(v.w); acc[q][7] += bf16_hi(v.w);
+                    }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int c = c0 + q * 32 + lane;
+                if (c < vec_per_row) {
+                    uint4 o;
+                    o.x = pack_bf16x2(acc[q][0], acc[q][1]);
+                    o.y = pack_bf16x2(acc[q][2], acc[q][3]);
+                    o.z = pack_bf16x2(acc[q][4], acc[q][5]);
+                    o.w = pack_bf16x2(acc[q][6], acc[q][7]);
+                    Y[(size_t)t * vec_per_row + c] = o;
+                }
+            }
+        }
+    }
+}
+
+// dgate[a] = sum over n-tiles of the partial dot products written by the dgrad-down epilogue
+// (row p = perm_row[a]; fixed order, so the result is reproducible).
+__global__ void dgate_reduce_kernel(const float* __restrict__ part, const int32_t* __restrict__ perm_row,
+                                    float* __restrict__ dgate, int M, int ntiles) {
+    const int a = blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= M) return;
+    const int32_t p = perm_row[a];
+    float s = 0.0f;
+    if (p >= 0)
+        for (int n = 0; n < ntiles; ++n) s += part[(size_t)n * M + p];
+    dgate[a] = s;
+}
+
+}  // namespace mop

@@ -1,0 +1,182 @@
+"""Parity of the CUDA path (called through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Integers (top-k indices, counts, offsets, permutation) must match bit for bit.  Floats: relative
+Frobenius error <= 1e-2 against the oracle's exact mode and max-abs error <= 2e-2 against its
+declared-rounding mode (bf16 roundings at the tensors the interface declares bf16), per tensor.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_01844_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+REL_FRO = 1e-2
+MAX_ABS = 2e-2
+
+
+def to_dev(host):
+    return {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in host.items()}
+
+
+def np_bias(host):
+    return None if host["bias"] is None else host["bias"].cpu().numpy()
+
+
+def run(w, gemm_path=binding.GEMM_AUTO, host=None):
+    host = host or synth.make_inputs(w, "cpu")
+    inp = to_dev(host)
+    ctx = binding.context_for(w, gemm_path=gemm_path)
+    buf = binding.LayerBuffers(w)
+    binding.forward(ctx, inp, buf)
+    if w.backward:
+        binding.backward(ctx, inp, buf)
+    binding.mop_poll(ctx)
+    torch.cuda.synchronize()
+    return host, inp, ctx, buf
+
+
+def rel_fro(got, ref):
+    n = np.linalg.norm(ref.astype(np.float64))
+    return float(np.linalg.norm(got.astype(np.float64) - ref.astype(np.float64)) / (n if n > 0 else 1.0))
+
+
+def check_float(name, got, exact, declared, max_abs=MAX_ABS):
+    r = rel_fro(got, exact)
+    m = float(np.max(np.abs(got.astype(np.float64) - declared.astype(np.float64)))) if got.size else 0.0
+    assert r <= REL_FRO, f"{name}: relative Frobenius error {r:.3e} vs exact oracle"
+    assert m <= max_abs, f"{name}: max-abs error {m:.3e} vs declared-rounding oracle"
+    return r, m
+
+
+def check_integers(w, host, buf):
+    xb = synth.bits(host["x"])
+    idx, gate = oracle.route(xb, host["W_r"].numpy(), np_bias(host), w.k, w.score_fn, w.bias_mode)
+    assert np.array_equal(buf.idx.cpu().numpy(), idx), "top-k indices"
+    g = buf.gate.cpu().numpy()
+    assert np.all(np.abs(g - gate) <= 1e-6 + 1e-5 * np.abs(gate)), "gates"
+    counts, offsets, perm_row, row_src = oracle.permute(idx, w.E)
+    assert np.array_equal(buf.counts.cpu().numpy(), counts), "counts"
+    assert np.array_equal(buf.offsets.cpu().numpy(), offsets), "offsets"
+    assert np.array_equal(buf.perm_row.cpu().numpy(), perm_row), "perm_row"
+    assert np.array_equal(buf.row_src.cpu().numpy(), row_src), "row_src"
+    Xp = synth.bits(buf.Xp)
+    assert np.array_equal(Xp, xb[row_src // w.k]), "Xp rows"
+    return idx, g
+
+
+def check_layer(w, gemm_path):
+    host, inp, ctx, buf = run(w, gemm_path)
+    idx, gate = check_integers(w, host, buf)   # the float checks use the CUDA path's gates (<= 1e-5 apart)
+    xb, Wg, Wu, Wd = (synth.bits(host[n]) for n in ("x", "W_gate", "W_up", "W_down"))
+    Y_e = oracle.ffn_fwd(xb, idx, gate, Wg, Wu, Wd)
+    Y_d = oracle.ffn_fwd(xb, idx, gate, Wg, Wu, Wd, declared=True)
+    check_float("Y", buf.Y.float().cpu().numpy(), Y_e, Y_d)
+    if w.backward:
+        dYb = synth.bits(host["dY"])
+        ex = np.arange(w.E, dtype=np.int32)
+        dX_e, dg_e = oracle.ffn_bwd_tokens(xb, dYb, idx, gate, Wg, Wu, Wd)
+        dX_d, dg_d = oracle.ffn_bwd_tokens(xb, dYb, idx, gate, Wg, Wu, Wd, declared=True)
+        dW_e = oracle.ffn_bwd_experts(xb, dYb, idx, gate, Wg, Wu, Wd, ex)
+        dW_d = oracle.ffn_bwd_experts(xb, dYb, idx, gate, Wg, Wu, Wd, ex, declared=True)
+        # magnitudes of dW and dgate grow with d and the row count, so their absolute bound is scaled
+        # by the largest reference value (the bound is 2e-2 where |ref| <= 1)
+        scale = lambda a: MAX_ABS * max(1.0, float(np.abs(a).max()))
+        check_float("dX", buf.dX.float().cpu().numpy(), dX_e, dX_d, scale(dX_d))
+        check_float("dgate", buf.dgate.cpu().numpy(), dg_e, dg_d, scale(dg_d))
+        for name, got, e, dd in zip(("dW_gate", "dW_up", "dW_down"), (buf.dW_gate, buf.dW_up, buf.dW_down), dW_e,
+                                    dW_d):
+            check_float(name, got.cpu().numpy(), e, dd, scale(dd))
+    return ctx, buf
+
+
+SMALL = [
+    synth.WORKLOADS["c1_tiny"],
+    synth.small("c1_tiny", backward=True),
+    synth.small("c2_mid", T=300, d=192, E=12, k=3, f=320, backward=True, seed=11),          # ragged tiles
+    synth.small("c3_trillion", T=200, d=256, E=40, k=8, f=128, backward=True, seed=12),     # sigmoid + bias
+    synth.small("c3_trillion", T=130, d=64, E=33, k=1, f=64, bias_mode=2, backward=True, seed=13),
+    synth.small("c1_tiny", T=64, d=128, E=4, k=4, f=64, backward=True, seed=14),            # k = E
+    synth.small("c1_tiny", T=1, d=64, E=3, k=2, f=64, backward=True, seed=15),              # one token
+    synth.small("c1_tiny", T=77, d=72, E=5, k=2, f=40, backward=True, seed=16),             # d, f multiples of 8 only
+]
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: f"{w.name}-T{w.T}d{w.d}E{w.E}k{w.k}f{w.f}{'b' if w.backward else ''}")
+@pytest.mark.parametrize("path", [binding.GEMM_SCALAR, binding.GEMM_AUTO], ids=["scalar", "auto"])
+def test_small_layers_match_oracle(w, path):
+    check_layer(w, path)
+
+
+def test_all_keys_equal_goes_to_lowest_ids_and_leaves_experts_empty():
+    w = synth.small("c1_tiny", T=96, d=64, E=6, k=2, f=64, backward=True, seed=17)
+    host = synth.make_inputs(w, "cpu")
+    host["W_r"] = torch.zeros_like(host["W_r"])
+    host, inp, ctx, buf = run(w, host=host)
+    assert np.array_equal(buf.idx.cpu().numpy(), np.tile(np.arange(2, dtype=np.int32), (96, 1)))
+    assert np.array_equal(buf.counts.cpu().numpy(), np.array([96, 96, 0, 0, 0, 0], np.int32))
+    assert torch.all(buf.dW_gate[2:] == 0) and torch.all(buf.dW_down[2:] == 0)
+    check_integers(w, host, buf)
+
+
+def test_zero_tokens_is_a_no_op():
+    w = synth.small("c1_tiny", T=0, d=64, E=4, k=2, f=64, backward=True)
+    host, inp, ctx, buf = run(w)
+    assert torch.all(buf.offsets == 0) and torch.all(buf.counts == 0)
+    assert torch.all(buf.dW_gate == 0) and torch.all(buf.dW_up == 0) and torch.all(buf.dW_down == 0)
+
+
+def test_results_are_bitwise_reproducible():
+    w = synth.small("c2_mid", T=512, d=256, E=16, k=4, f=256, backward=True, seed=18)
+    _, _, _, a = run(w)
+    _, _, _, b = run(w)
+    for n in ("idx", "gate", "perm_row", "Xp", "H", "Yp", "Y", "dX", "dgate", "dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(getattr(a, n), getattr(b, n)), n
+
+
+def test_dw_accumulate_adds_into_existing_gradients():
+    w = synth.small("c1_tiny", T=128, d=64, E=4, k=2, f=64, backward=True, seed=19)
+    host = synth.make_inputs(w, "cpu")
+    inp = to_dev(host)
+    ctx = binding.context_for(w, dw_accumulate=True)
+    buf = binding.LayerBuffers(w)
+    for t in (buf.dW_gate, buf.dW_up, buf.dW_down):
+        t.fill_(1.0)
+    binding.forward(ctx, inp, buf)
+    binding.backward(ctx, inp, buf)
+    _, _, _, ref = run(w, host=host)
+    for n in ("dW_gate", "dW_up", "dW_down"):
+        assert torch.allclose(getattr(buf, n), getattr(ref, n) + 1.0, atol=1e-5), n
+
+
+def test_bad_arguments_return_codes():
+    w = synth.WORKLOADS["c1_tiny"]
+    ctx = binding.context_for(w)
+    buf = binding.LayerBuffers(w)
+    with pytest.raises(binding.MopError) as e:
+        binding.mop_moe_combine(ctx, None, buf.perm_row, buf.Y)
+    assert e.value.code == 1
+    with pytest.raises(binding.MopError) as e:
+        binding.mop_moe_combine(ctx, buf.Yp.data_ptr() + 2, buf.perm_row, buf.Y)
+    assert e.value.code == 3
+    with pytest.raises(binding.MopError) as e:   # backward on a forward-only context
+        binding.mop_moe_expert_ffn_bwd(ctx, *([buf.Yp] * 17))
+    assert e.value.code == 6
+    with pytest.raises(binding.MopError) as e:
+        binding.Context(16, 64, 4, 5, 64)
+    assert e.value.code == 1
+
+
+def test_forward_host_entry_point_matches_device_path():
+    w = synth.small("c2_mid", T=256, d=128, E=8, k=2, f=192, seed=20)
+    host, inp, _, buf = run(w)
+    ctx = binding.context_for(w, host_io=True)
+    xh = host["x"].pin_memory()
+    Yh = torch.empty_like(xh).pin_memory()
+    idxh = torch.empty((w.T, w.k), dtype=torch.int32).pin_memory()
+    gh = torch.empty((w.T, w.k), dtype=torch.float32).pin_memory()
+    binding.mop_moe_forward_host(ctx, xh, inp["W_r"], inp["bias"], inp["W_gate"], inp["W_up"], inp["W_down"], Yh, idxh,
+                                 gh)
+    assert torch.equal(Yh, buf.Y.cpu()) and torch.equal(idxh, buf.idx.cpu()) and torch.equal(gh, buf.gate.cpu())
