@@ -56,7 +56,7 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_permute.argtypes = [_P] * 9
         L.mop_moe_expert_ffn_fwd.argtypes = [_P] * 13
         L.mop_moe_combine.argtypes = [_P] * 5
-        L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 20
+        L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 19
         L.mop_moe_forward_host.argtypes = [_P] * 11
         _lib = L
     return _lib

@@ -62,6 +62,8 @@ def _gen(seed: int, stream: int, device) -> torch.Generator:
 def _normal_bf16(shape, std, gen, device, chunk_rows=None):
     """N(0, std) drawn in fp32 and rounded once to bf16, in slabs to bound temporaries."""
     out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    if out.numel() == 0:
+        return out
     flat = out.view(shape[0], -1)
     step = chunk_rows or max(1, (1 << 28) // max(1, flat.shape[1]))
     for r0 in range(0, flat.shape[0], step):
