@@ -1,11 +1,506 @@
-// Tensor-core (tcgen05 / TMEM / TMA) grouped GEMMs -- interface.
+// Tensor-core grouped GEMMs for sm_100a: tcgen05.mma with TMEM accumulators, operands staged by
+// TMA into 128-byte-swizzled shared memory, one persistent warp-specialised CTA per SM.
+//
+// Every GEMM of the layer is one instantiation of tc_grouped_gemm_kernel<KIND>:
+//   F1   [G|U] = Xp W_gate[e] | Xp W_up[e]        SwiGLU epilogue -> H (+ stash)      ragged M
+//   F2   O     = H W_down[e]                      gate epilogue   -> Yp               ragged M
+//   B2   dHu   = dYp W_down[e]^T                  SwiGLU-backward epilogue            ragged M
+//   B4   dXp   = dG W_gate[e]^T + dU W_up[e]^T    (two K phases)  -> bf16             ragged M
+//   WD   dW_down[e] = (gate H)_e^T dYp_e          fp32 store                          ragged K
+//   WGU  [dW_gate|dW_up][e] = Xp_e^T [dG|dU]_e    fp32 store                          ragged K
+// CTA tile 128 x 256 (one tcgen05.mma.cta_group::1 of M=128, N=256, K=16 per 32 bytes of K),
+// K step 64 per pipeline stage, 4 stages, two 256-column accumulators in TMEM so that the
+// epilogue of tile i overlaps the main loop of tile i+1.
+//
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2..5 = epilogue.
+// Every mbarrier wait is bounded: on expiry the CTA records a code in the status word, raises a
+// CTA-wide abort flag, lets its copies land, frees TMEM and returns.
 #pragma once
+#include <cuda.h>
+
 #include "../../include/mop_moe.h"
 #include "epilogue.cuh"
 
 namespace mop {
 
-struct TcPlan { int sm_count; mop_moe_shape s; };
+enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5 };
+
+constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64, TC_STAGES = 4;
+constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // 16 KiB
+constexpr int TC_B_BYTES = TC_BN * TC_BK * 2;   // 32 KiB
+constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
+constexpr int TC_CHUNK_BYTES = 64 * TC_BK * 2;  // one 64-wide MN chunk of 64 K rows: 8 KiB
+constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int TC_THREADS = 192;
+constexpr long long TC_WAIT_CYCLES = 4000000000ll;  // about two seconds
+
+template <int KIND>
+struct TcTraits {
+    static constexpr bool A_MN = (KIND == TC_WD || KIND == TC_WGU);   // A is M-contiguous in memory
+    static constexpr bool B_MN = (KIND != TC_B2 && KIND != TC_B4);    // B is N-contiguous in memory
+    static constexpr bool DUAL_B = (KIND == TC_F1 || KIND == TC_WGU); // two B tensors, 128 columns each
+    static constexpr bool RAGGED_K = A_MN;
+    static constexpr bool B_WEIGHT = !RAGGED_K;                       // B is an [E, ., .] weight tensor
+    static constexpr int PHASES = (KIND == TC_B4) ? 2 : 1;
+    static constexpr int N_PER_TILE = DUAL_B ? 128 : 256;             // output columns per tensor per tile
+};
+
+struct TcArgs {
+    const int32_t* offsets;
+    const int4* mtiles;      // ragged M: {expert, first row, rows, 0} per 128-row tile
+    const int32_t* n_mtiles; // device scalar
+    int E;
+    int tiles_n;             // n-tiles per row block
+    int tiles_m_fixed;       // ragged K: m-tiles per expert
+    int kblocks;             // ragged M: K / 64 (rounded up) per phase
+    int Mfix, N;             // ragged K: output rows per expert; N = columns per output tensor
+    int32_t* status;
+    EpiArgs ep;
+    float* outf1;            // WGU: second output tensor
+};
+
+// ------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > TC_WAIT_CYCLES) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+}
+
+// Warp-uniform form: lane 0 waits, the verdict is broadcast, and every lane then observes the
+// completed phase itself (so that its later reads are ordered after the barrier).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* status, int code, int lane) {
+    uint32_t ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, status, code) ? 1u : 0u;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (ok) (void)mbar_try_wait(bar, parity);
+    return ok != 0;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], "
+        "[%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(
+            d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets lane (base lane + i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, version 1 (Blackwell).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 operands, M=128, N=256, operand majors.
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------ tiles
+struct TileInfo {
+    int e, row0, rows;   // ragged M: first global row and valid rows; ragged K: first k row and k count
+    int m0;              // ragged K: first output row of the tile inside the expert's matrix
+    int nt;              // n-tile index
+    bool skip;           // nothing to multiply (expert without rows)
+};
+
+template <int KIND>
+__device__ __forceinline__ TileInfo decode_tile(const TcArgs& a, int t) {
+    TileInfo ti;
+    if constexpr (TcTraits<KIND>::RAGGED_K) {
+        const int per_e = a.tiles_m_fixed * a.tiles_n;
+        ti.e = t / per_e;
+        const int r = t - ti.e * per_e;
+        ti.m0 = (r / a.tiles_n) * TC_BM;
+        ti.nt = r % a.tiles_n;
+        ti.row0 = a.offsets[ti.e];
+        ti.rows = a.offsets[ti.e + 1] - ti.row0;
+        ti.skip = ti.rows <= 0;
+    } else {
+        const int4 m = a.mtiles[t / a.tiles_n];
+        ti.e = m.x; ti.row0 = m.y; ti.rows = m.z; ti.m0 = 0;
+        ti.nt = t % a.tiles_n;
+        ti.skip = false;
+    }
+    return ti;
+}
+
+// 128-row tile list of the ragged-M GEMMs, built on the device from offsets (no host round trip).
+__global__ void __launch_bounds__(1024) tc_build_mtiles_kernel(const int32_t* __restrict__ offsets, int E,
+                                                               int4* __restrict__ mtiles,
+                                                               int32_t* __restrict__ n_mtiles) {
+    __shared__ int32_t scan[1025];
+    const int e = threadIdx.x;
+    int cnt = 0, off = 0;
+    if (e < E) { off = offsets[e]; cnt = offsets[e + 1] - off; }
+    const int nt = (cnt + TC_BM - 1) / TC_BM;
+    scan[e] = nt;
+    __syncthreads();
+    // inclusive scan, Hillis-Steele over 1024 entries
+    for (int s = 1; s < 1024; s <<= 1) {
+        const int v = (e >= s) ? scan[e - s] : 0;
+        __syncthreads();
+        scan[e] += v;
+        __syncthreads();
+    }
+    const int first = scan[e] - nt;
+    for (int i = 0; i < nt; ++i) mtiles[first + i] = make_int4(e, off + i * TC_BM, min(TC_BM, cnt - i * TC_BM), 0);
+    if (e == 1023) *n_mtiles = scan[1023];
+}
+
+// ------------------------------------------------------------------------------------------ kernel
+template <int KIND>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
+                       const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
+                       const TcArgs args) {
+    using Tr = TcTraits<KIND>;
+    extern __shared__ uint8_t tc_smem_raw[];
+    // 1024-byte alignment: the swizzle pattern is a function of address bits 7..9
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + TC_STAGES * TC_STAGE_BYTES);
+    // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_STAGES + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (TC_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * TC_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * TC_STAGES + 2 + b); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB0);
+        if (Tr::PHASES == 2) tma_prefetch_desc(&tmA1);
+        if (Tr::DUAL_B || Tr::PHASES == 2) tma_prefetch_desc(&tmB1);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    int total_tiles;
+    if constexpr (Tr::RAGGED_K) total_tiles = args.E * args.tiles_m_fixed * args.tiles_n;
+    else total_tiles = (*args.n_mtiles) * args.tiles_n;
+
+    if (warp == 0) {
+        // ===================================================================== TMA producer
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool alive = true;
+            for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+                const TileInfo ti = decode_tile<KIND>(args, t);
+                if (ti.skip) continue;
+                const int n0 = ti.nt * Tr::N_PER_TILE;
+                const int nkb = Tr::RAGGED_K ? (ti.rows + TC_BK - 1) / TC_BK : Tr::PHASES * args.kblocks;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) {
+                        alive = false; break;
+                    }
+                    const uint32_t fb = full_bar(stage);
+                    mbar_expect_tx(fb, TC_STAGE_BYTES);
+                    const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
+                    const uint32_t sB = sA + TC_A_BYTES;
+                    const int ph = (Tr::PHASES == 2 && kb >= args.kblocks) ? 1 : 0;
+                    const int k0 = (kb - ph * args.kblocks) * TC_BK;
+                    if constexpr (!Tr::A_MN) {
+                        tma_load_2d(sA, ph ? &tmA1 : &tmA0, fb, k0, ti.row0);
+                    } else {
+                        const int krow = ti.row0 + kb * TC_BK;
+                        tma_load_2d(sA, &tmA0, fb, ti.m0, krow);
+                        tma_load_2d(sA + TC_CHUNK_BYTES, &tmA0, fb, ti.m0 + 64, krow);
+                    }
+                    if constexpr (!Tr::B_MN) {
+                        tma_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0, n0, ti.e);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const CUtensorMap* mp = (Tr::DUAL_B && c >= 2) ? &tmB1 : &tmB0;
+                            const int n = Tr::DUAL_B ? n0 + 64 * (c & 1) : n0 + 64 * c;
+                            if constexpr (Tr::B_WEIGHT) tma_load_3d(sB + c * TC_CHUNK_BYTES, mp, fb, n, k0, ti.e);
+                            else tma_load_2d(sB + c * TC_CHUNK_BYTES, mp, fb, n, ti.row0 + kb * TC_BK);
+                        }
+                    }
+                    if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================================================================== MMA issuer
+        constexpr uint32_t idesc = make_idesc(Tr::A_MN, Tr::B_MN);
+        // MN-major operand: 64-wide chunks are TC_CHUNK_BYTES apart (leading offset), groups of
+        // 8 K rows are 1024 bytes apart (stride offset); K-major: 8-row groups 1024 bytes apart.
+        constexpr uint32_t mn_lbo = TC_CHUNK_BYTES, mn_sbo = 1024u;
+        int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
+        for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+            const TileInfo ti = decode_tile<KIND>(args, t);
+            if (ti.skip) continue;
+            const int buf = it & 1;
+            const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
+            if (!mbar_wait_warp(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY, lane)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)buf * TC_BN;
+            const int nkb = Tr::RAGGED_K ? (ti.rows + TC_BK - 1) / TC_BK : Tr::PHASES * args.kblocks;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!mbar_wait_warp(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL, lane)) {
+                    alive = false; break;
+                }
+                tc_fence_after();
+                const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
+                const uint32_t sB = sA + TC_A_BYTES;
+                if constexpr (Tr::RAGGED_K) {
+                    // K tail: rows past the expert's end belong to the next expert -> zero them
+                    const int valid = ti.rows - kb * TC_BK;
+                    if (valid < TC_BK) {
+                        uint8_t* base = smem + stage * TC_STAGE_BYTES;
+                        const int nrows = TC_BK - valid;
+                        for (int i = lane; i < 6 * nrows * 8; i += 32) {
+                            const int chunk = i / (nrows * 8), rem = i % (nrows * 8);
+                            const int row = valid + rem / 8, v = rem % 8;
+                            *reinterpret_cast<uint4*>(base + chunk * TC_CHUNK_BYTES + row * 128 + v * 16) =
+                                make_uint4(0, 0, 0, 0);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
+                if (lane == 0) {
+#pragma unroll
+                    for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
+                        const uint64_t ad = Tr::A_MN ? smem_desc(sA + k4 * 2048, mn_lbo, mn_sbo)
+                                                     : smem_desc(sA + k4 * 32, 0, 1024);
+                        const uint64_t bd = Tr::B_MN ? smem_desc(sB + k4 * 2048, mn_lbo, mn_sbo)
+                                                     : smem_desc(sB + k4 * 32, 0, 1024);
+                        umma_bf16(d_tmem, ad, bd, idesc, (kb | k4) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));
+                }
+                __syncwarp();
+                if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!alive) break;
+            if (lane == 0) umma_commit(tfull_bar(buf));
+            __syncwarp();
+            ++it;
+        }
+    } else {
+        // ===================================================================== epilogue (4 warps)
+        const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int r = quarter * 32 + lane;       // row of the tile owned by this thread
+        int it = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            const TileInfo ti = decode_tile<KIND>(args, t);
+            const int n0 = ti.nt * Tr::N_PER_TILE;
+            if constexpr (Tr::RAGGED_K) {
+                if (ti.skip) {
+                    // expert without rows: its gradient is zero (or unchanged when accumulating)
+                    if (!args.ep.accumulate && ti.m0 + r < args.Mfix) {
+                        const size_t ro = ((size_t)ti.e * args.Mfix + ti.m0 + r) * args.N;
+                        for (int c = 0; c < TC_BN; c += 4) {
+                            const int cc = Tr::DUAL_B ? (c & 127) : c;
+                            float* dst = (Tr::DUAL_B && c >= 128) ? args.outf1 : args.ep.outf;
+                            if (n0 + cc < args.N) *reinterpret_cast<float4*>(dst + ro + n0 + cc) = make_float4(0, 0, 0, 0);
+                        }
+                    }
+                    continue;
+                }
+            }
+            const int buf = it & 1;
+            const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
+            if (!mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * TC_BN;
+            const bool row_ok = Tr::RAGGED_K ? (ti.m0 + r < args.Mfix) : (r < ti.rows);
+            const int grow = ti.row0 + r;        // ragged M: global row
+            float acc[32];
+
+            if constexpr (KIND == TC_F1) {
+                float acc2[32];
+#pragma unroll 1
+                for (int c = 0; c < 128; c += 32) {
+                    tmem_ld32(taddr + c, acc);
+                    tmem_ld32(taddr + 128 + c, acc2);
+                    if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                        for (int s = 0; s < 32; s += 8) {
+                            float g8[8], u8[8];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) { g8[q] = acc[s + q]; u8[q] = acc2[s + q]; }
+                            epi_swiglu<8>(args.ep, grow, n0 + c + s, g8, u8);
+                        }
+                    }
+                }
+            } else if constexpr (KIND == TC_F2 || KIND == TC_B2) {
+                const float gate = row_ok ? args.ep.gate[args.ep.row_src[grow]] : 0.0f;
+                float dot = 0.0f;
+#pragma unroll 1
+                for (int c = 0; c < TC_BN; c += 32) {
+                    tmem_ld32(taddr + c, acc);
+                    if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                        for (int s = 0; s < 32; s += 8) {
+                            float a8[8];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
+                            if constexpr (KIND == TC_F2) epi_gate<8>(args.ep, grow, n0 + c + s, gate, a8);
+                            else dot += epi_dh<8>(args.ep, grow, n0 + c + s, gate, a8);
+                        }
+                    }
+                }
+                if (KIND == TC_B2 && row_ok) args.ep.part[(size_t)ti.nt * args.ep.M_total + grow] = dot;
+            } else if constexpr (KIND == TC_B4) {
+#pragma unroll 1
+                for (int c = 0; c < TC_BN; c += 32) {
+                    tmem_ld32(taddr + c, acc);
+                    if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                        for (int s = 0; s < 32; s += 8) {
+                            float a8[8];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
+                            store_bf16_run<8>(args.ep.out0 + (size_t)grow * args.ep.ldo + n0 + c + s, a8);
+                        }
+                    }
+                }
+            } else {
+                const size_t ro = ((size_t)ti.e * args.Mfix + ti.m0 + r) * args.N;
+#pragma unroll 1
+                for (int c = 0; c < TC_BN; c += 32) {
+                    tmem_ld32(taddr + c, acc);
+                    const int cc = Tr::DUAL_B ? (c & 127) : c;
+                    float* dst = (Tr::DUAL_B && c >= 128) ? args.outf1 : args.ep.outf;
+                    if (row_ok && n0 + cc < args.N) {
+#pragma unroll
+                        for (int s = 0; s < 32; s += 8) {
+                            float a8[8];
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
+                            epi_f32<8>(dst + ro + n0 + cc + s, a8, args.ep.accumulate);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            ++it;
+        }
+    }
+
+    // ------------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // let copies that are still in flight land before the shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host
+struct TcPlan {
+    int sm_count;
+    mop_moe_shape s;
+    void* encode;   // cuTensorMapEncodeTiled
+};
 
 struct TcFwdArgs {
     const bf16* Xp; const int32_t* offsets; const int32_t* row_src; const float* gate;
@@ -20,10 +515,170 @@ struct TcBwdArgs {
     float *dW_gate, *dW_up, *dW_down; int accumulate;
 };
 
-inline bool tc_shape_supported(int d, int f) { (void)d; (void)f; return false; }
-inline size_t tc_tile_table_bytes(int M, int E) { (void)M; (void)E; return 256; }
-inline mop_status tc_plan_init(TcPlan*, const mop_moe_shape&, int) { return MOP_OK; }
-inline mop_status tc_ffn_fwd(TcPlan*, const TcFwdArgs&, int32_t*, int32_t*, cudaStream_t, int*) { return MOP_ERR_UNSUPPORTED; }
-inline mop_status tc_ffn_bwd(TcPlan*, const TcBwdArgs&, int32_t*, int32_t*, cudaStream_t, int*, int*) { return MOP_ERR_UNSUPPORTED; }
+inline bool tc_shape_supported(int d, int f) { return d % 64 == 0 && f % 64 == 0; }
+inline size_t tc_tile_table_bytes(int M, int E) { return ((size_t)M / TC_BM + E + 8) * sizeof(int4) + 256; }
+
+typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+template <int KIND>
+inline mop_status tc_set_smem() {
+    return cudaFuncSetAttribute(tc_grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                TC_SMEM_BYTES) == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count) {
+    p->sm_count = sm_count;
+    p->s = s;
+    cudaDriverEntryPointQueryResult q;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+        q != cudaDriverEntryPointSuccess)
+        return MOP_ERR_CUDA;
+    p->encode = fn;
+    mop_status r;
+    if ((r = tc_set_smem<TC_F1>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_F2>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_B2>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_B4>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_WD>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_WGU>()) != MOP_OK) return r;
+    return MOP_OK;
+}
+
+// 2-D map over a dense [rows, cols] bf16 matrix; box = {64 cols, box_rows}.
+inline bool tc_map_2d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                      uint32_t box_rows) {
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t es[2] = {1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// 3-D map over a dense [E, rows, cols] bf16 tensor; box = {64 cols, box_rows, 1}.
+inline bool tc_map_3d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows, uint64_t cols,
+                      uint32_t box_rows) {
+    const cuuint64_t dims[3] = {cols, rows, E};
+    const cuuint64_t strides[2] = {cols * 2, rows * cols * 2};
+    const cuuint32_t box[3] = {64, box_rows, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int KIND>
+inline mop_status tc_launch(const TcPlan* p, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
+                            const CUtensorMap& b1, const TcArgs& args, cudaStream_t st) {
+    tc_grouped_gemm_kernel<KIND><<<p->sm_count, TC_THREADS, TC_SMEM_BYTES, st>>>(a0, a1, b0, b1, args);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+inline TcArgs tc_base_args(const TcPlan* p, const int32_t* offsets, int32_t* tiles, int32_t* status) {
+    TcArgs a{};
+    a.offsets = offsets;
+    a.n_mtiles = tiles;                                   // first word of the table area
+    a.mtiles = reinterpret_cast<const int4*>(tiles + 64); // entries start 256 bytes in
+    a.E = p->s.E;
+    a.status = status;
+    return a;
+}
+
+inline mop_status tc_build_tiles(const TcPlan* p, const int32_t* offsets, int32_t* tiles, cudaStream_t st) {
+    tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(offsets, p->s.E, reinterpret_cast<int4*>(tiles + 64), tiles);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
+                             int* launches) {
+    const mop_moe_shape& s = p->s;
+    const uint64_t M = (uint64_t)s.T * s.k;
+    mop_status r;
+    if ((r = tc_build_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
+    ++*launches;
+    CUtensorMap mXp, mWg, mWu, mH, mWd;
+    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, 128) || !tc_map_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 64) ||
+        !tc_map_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 64) || !tc_map_2d(p, &mH, a.H, M, s.f, 128) ||
+        !tc_map_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 64))
+        return MOP_ERR_CUDA;
+    {   // F1: [G|U] = Xp [W_gate | W_up], SwiGLU epilogue
+        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
+        g.tiles_n = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
+        g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
+        if ((r = tc_launch<TC_F1>(p, mXp, mXp, mWg, mWu, g, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    {   // F2: Yp = gate * (H W_down)
+        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
+        g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
+        g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
+        if ((r = tc_launch<TC_F2>(p, mH, mH, mWd, mWd, g, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    return MOP_OK;
+}
+
+inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
+                             int* launches, int* ntile_part) {
+    const mop_moe_shape& s = p->s;
+    const uint64_t M = (uint64_t)s.T * s.k;
+    *ntile_part = ceil_div(s.f, 256);
+    if (M == 0) {
+        // no rows at all: gradients are zero unless accumulating
+        if (!a.accumulate) {
+            const size_t n = (size_t)s.E * s.d * s.f * 4;
+            if (cudaMemsetAsync(a.dW_gate, 0, n, st) != cudaSuccess || cudaMemsetAsync(a.dW_up, 0, n, st) != cudaSuccess ||
+                cudaMemsetAsync(a.dW_down, 0, n, st) != cudaSuccess)
+                return MOP_ERR_CUDA;
+        }
+        return MOP_OK;
+    }
+    mop_status r;
+    if ((r = tc_build_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
+    ++*launches;
+    CUtensorMap mdYpA, mWdK, mdG, mdU, mWgK, mWuK, mgH, mdYpB, mXpA, mdGB, mdUB;
+    if (!tc_map_2d(p, &mdYpA, a.dYp, M, s.d, 128) || !tc_map_3d(p, &mWdK, a.W_down, s.E, s.f, s.d, 256) ||
+        !tc_map_2d(p, &mdG, a.dG, M, s.f, 128) || !tc_map_2d(p, &mdU, a.dU, M, s.f, 128) ||
+        !tc_map_3d(p, &mWgK, a.W_gate, s.E, s.d, s.f, 256) || !tc_map_3d(p, &mWuK, a.W_up, s.E, s.d, s.f, 256) ||
+        !tc_map_2d(p, &mgH, a.gH, M, s.f, 64) || !tc_map_2d(p, &mdYpB, a.dYp, M, s.d, 64) ||
+        !tc_map_2d(p, &mXpA, a.Xp, M, s.d, 64) || !tc_map_2d(p, &mdGB, a.dG, M, s.f, 64) ||
+        !tc_map_2d(p, &mdUB, a.dU, M, s.f, 64))
+        return MOP_ERR_CUDA;
+    {   // B2: dHu = dYp W_down^T, SwiGLU backward epilogue
+        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
+        g.tiles_n = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
+        g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
+        g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.part = a.part; g.ep.ldo = s.f; g.ep.M_total = (int)M;
+        if ((r = tc_launch<TC_B2>(p, mdYpA, mdYpA, mWdK, mWdK, g, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    {   // B4: dXp = dG W_gate^T + dU W_up^T
+        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
+        g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
+        g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
+        if ((r = tc_launch<TC_B4>(p, mdG, mdU, mWgK, mWuK, g, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    {   // WD: dW_down[e] = (gate H)_e^T dYp_e
+        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
+        g.tiles_n = ceil_div(s.d, 256); g.tiles_m_fixed = ceil_div(s.f, TC_BM); g.Mfix = s.f; g.N = s.d;
+        g.ep.outf = a.dW_down; g.ep.accumulate = a.accumulate;
+        if ((r = tc_launch<TC_WD>(p, mgH, mgH, mdYpB, mdYpB, g, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    {   // WGU: [dW_gate | dW_up][e] = Xp_e^T [dG | dU]_e
+        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
+        g.tiles_n = ceil_div(s.f, 128); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
+        g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate;
+        if ((r = tc_launch<TC_WGU>(p, mXpA, mXpA, mdGB, mdUB, g, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    return MOP_OK;
+}
 
 }  // namespace mop

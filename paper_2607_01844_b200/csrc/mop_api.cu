@@ -108,7 +108,13 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
         if (!aligned16(p)) return MOP_ERR_ALIGN;        \
     } while (0)
 
-#define CUDA_OK(expr)                                   \
+// token-sized tensors may be null when the layer has no tokens (an empty tensor has no storage)
+#define REQ_PTR_T(p)                                    \
+    do {                                                \
+        if (c->s.T > 0) REQ_PTR(p);                     \
+    } while (0)
+
+#define CUDA_OK(expr)                                 \
     do {                                                \
         if ((expr) != cudaSuccess) return MOP_ERR_CUDA; \
     } while (0)
@@ -248,7 +254,7 @@ mop_status mop_poll(mop_ctx* c, void* stream) {
 mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const float* bias, int32_t* topk_idx,
                          float* topk_gate, float* logits_opt, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
-    REQ_PTR(x); REQ_PTR(W_r); REQ_PTR(topk_idx); REQ_PTR(topk_gate);
+    REQ_PTR_T(x); REQ_PTR(W_r); REQ_PTR_T(topk_idx); REQ_PTR_T(topk_gate);
     if ((c->s.bias_mode != MOP_BIAS_NONE) != (bias != nullptr)) return MOP_ERR_INVALID_ARG;
     if (logits_opt && !aligned16(logits_opt)) return MOP_ERR_ALIGN;
     const mop_moe_shape& s = c->s;
@@ -270,7 +276,8 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
 mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, int32_t* counts, int32_t* offsets,
                            int32_t* perm_row, int32_t* row_src, void* Xp, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
-    REQ_PTR(x); REQ_PTR(topk_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR(perm_row); REQ_PTR(row_src); REQ_PTR(Xp);
+    REQ_PTR_T(x); REQ_PTR_T(topk_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR_T(perm_row); REQ_PTR_T(row_src);
+    REQ_PTR_T(Xp);
     const mop_moe_shape& s = c->s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MOP_ERR_CUDA;
@@ -297,7 +304,7 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
 
 mop_status mop_moe_combine(mop_ctx* c, const void* Yp, const int32_t* perm_row, void* Y, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
-    REQ_PTR(Yp); REQ_PTR(perm_row); REQ_PTR(Y);
+    REQ_PTR_T(Yp); REQ_PTR_T(perm_row); REQ_PTR_T(Y);
     const mop_moe_shape& s = c->s;
     if (s.T == 0) return MOP_OK;
     DeviceGuard guard(c->device);
@@ -312,8 +319,8 @@ mop_status mop_moe_expert_ffn_fwd(mop_ctx* c, const void* Xp, const int32_t* off
                                   const float* topk_gate, const void* W_gate, const void* W_up, const void* W_down,
                                   void* G_save, void* U_save, void* H, void* Yp, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
-    REQ_PTR(Xp); REQ_PTR(offsets); REQ_PTR(row_src); REQ_PTR(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up);
-    REQ_PTR(W_down); REQ_PTR(H); REQ_PTR(Yp);
+    REQ_PTR_T(Xp); REQ_PTR(offsets); REQ_PTR_T(row_src); REQ_PTR_T(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up);
+    REQ_PTR(W_down); REQ_PTR_T(H); REQ_PTR_T(Yp);
     if ((G_save == nullptr) != (U_save == nullptr)) return MOP_ERR_INVALID_ARG;
     if (G_save && (!aligned16(G_save) || !aligned16(U_save))) return MOP_ERR_ALIGN;
     const mop_moe_shape& s = c->s;
@@ -358,9 +365,9 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
                                   float* dW_down, float* dgate, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
     if (!c->s.with_backward) return MOP_ERR_UNSUPPORTED;
-    REQ_PTR(dY); REQ_PTR(Xp); REQ_PTR(G_save); REQ_PTR(U_save); REQ_PTR(H); REQ_PTR(offsets); REQ_PTR(perm_row);
-    REQ_PTR(row_src); REQ_PTR(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up); REQ_PTR(W_down); REQ_PTR(dX);
-    REQ_PTR(dW_gate); REQ_PTR(dW_up); REQ_PTR(dW_down); REQ_PTR(dgate);
+    REQ_PTR_T(dY); REQ_PTR_T(Xp); REQ_PTR_T(G_save); REQ_PTR_T(U_save); REQ_PTR_T(H); REQ_PTR(offsets);
+    REQ_PTR_T(perm_row); REQ_PTR_T(row_src); REQ_PTR_T(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up); REQ_PTR(W_down);
+    REQ_PTR_T(dX); REQ_PTR(dW_gate); REQ_PTR(dW_up); REQ_PTR(dW_down); REQ_PTR_T(dgate);
     const mop_moe_shape& s = c->s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MOP_ERR_CUDA;
