@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the routed-expert MoE layer on B200: one step = one pass of the whole hot path
+(route -> permute -> grouped SwiGLU GEMMs -> combine, plus the backward when the workload has one)
+over one batch of seeded synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is useful TFLOP/s of the whole job with inputs resident in
+HBM; `e2e` is the same metric through the host-buffer entry point of the C ABI (activations copied
+from / to pinned host memory inside the timed region); `roofline` is for the kernel that takes the
+largest share of the step; `cpu_baseline` is the CPU oracle timed on a bounded sample.
+With N > 1 every rank runs the same workload on its own GPU (the layer has no collective; weak
+scaling) and the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import numpy as np
+import torch
+
+from paper_2607_01844_b200 import synth
+
+# fallback denominators if MEASURED_PEAKS.json is absent (an earlier measurement on this machine)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
+# (kernel, workload).  Filled from the summaries under profiles/; None = not captured.
+NCU_TRAFFIC_BYTES: dict = {}
+
+
+def peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def flops_per_step(w):
+    return (18 if w.backward else 6) * w.M * w.d * w.f
+
+
+def kernel_work(w, counts):
+    """Algorithmic flops and bytes of one launch of each kernel (useful rows only, every tensor moved once)."""
+    T, d, E, k, f, M = w.T, w.d, w.E, w.k, w.f, w.M
+    live = int((counts > 0).sum())
+    mdf = M * d * f
+    stash = 3 if w.backward else 1
+    return {
+        "route_score": (2 * T * d * E, T * d * 2 + d * E * 4 + T * E * 4),
+        "route_select": (0, T * E * 4 + T * k * 8),
+        "permute_scatter_rows": (0, T * d * 2 + M * d * 2 + M * 4),
+        "dy_scatter_rows": (0, T * d * 2 + M * d * 2 + M * 4),
+        "combine_rows": (0, M * d * 2 + T * d * 2 + M * 4),
+        "gemm_up_swiglu": (4 * mdf, live * 2 * d * f * 2 + M * d * 2 + stash * M * f * 2),
+        "gemm_down_gate": (2 * mdf, live * d * f * 2 + M * f * 2 + M * d * 2),
+        "gemm_dgrad_down_dswiglu": (2 * mdf, live * d * f * 2 + M * d * 2 + 6 * M * f * 2),
+        "gemm_dgrad_gate_up": (4 * mdf, live * 2 * d * f * 2 + 2 * M * f * 2 + M * d * 2),
+        "gemm_wgrad_down": (2 * mdf, E * d * f * 4 + M * f * 2 + M * d * 2),
+        "gemm_wgrad_gate_up": (4 * mdf, 2 * E * d * f * 4 + M * d * 2 + 2 * M * f * 2),
+    }
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region (read-only query)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons, pw = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w": float(np.median(pw)) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_expert_sample(w, host_slices, n_experts, backward):
+    """Time the oracle, as it stands, on the complete work of `n_experts` experts of this workload
+    (every row routed to them: forward, and dgrad + wgrad when the workload has a backward).
+    Returns (seconds, useful flops, rows)."""
+    import oracle
+    secs, flops, rows_total = 0.0, 0, 0
+    for sl in host_slices[:n_experts]:
+        rows = sl["x"].shape[0]
+        if rows == 0:
+            continue
+        idx = np.zeros((rows, 1), np.int32)
+        gate = sl["gate"].reshape(rows, 1).astype(np.float32)
+        t0 = time.perf_counter()
+        if backward:
+            oracle.ffn_bwd_experts(sl["x"], sl["dY"], idx, gate, sl["Wg"], sl["Wu"], sl["Wd"], np.zeros(1, np.int32))
+            oracle.ffn_bwd_tokens(sl["x"], sl["dY"], idx, gate, sl["Wg"], sl["Wu"], sl["Wd"])
+        else:
+            oracle.ffn_fwd(sl["x"], idx, gate, sl["Wg"], sl["Wu"], sl["Wd"])
+        secs += time.perf_counter() - t0
+        flops += rows * (18 if backward else 6) * w.d * w.f
+        rows_total += rows
+    return secs, flops, rows_total
+
+
+def expert_slices(w, inp, idx, gate, experts):
+    """Host copies of everything the oracle needs for the listed experts (rows routed to them)."""
+    out = []
+    flat = idx.reshape(-1)
+    for e in experts:
+        a = torch.nonzero(flat == e).reshape(-1)
+        t = a // w.k
+        sl = {"x": synth.bits(inp["x"][t]), "gate": gate.reshape(-1)[a].float().cpu().numpy(),
+              "Wg": synth.bits(inp["W_gate"][e:e + 1]), "Wu": synth.bits(inp["W_up"][e:e + 1]),
+              "Wd": synth.bits(inp["W_down"][e:e + 1])}
+        if w.backward:
+            sl["dY"] = synth.bits(inp["dY"][t])
+        out.append(sl)
+    return out
+
+
+def run_reference(args, w):
+    """The oracle on the host cores: each step is a bounded sample (the complete work of one expert)."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    oracle.build()
+    dev = "cpu"
+    torch.manual_seed(0)
+    # inputs of the sampled experts only: same distributions, generated on the host
+    rows = max(1, w.M // w.E)
+    n_exp = args.steps + args.warmup
+    g = torch.Generator().manual_seed(w.seed)
+    def rnd(shape, std):
+        return synth.bits((torch.randn(shape, generator=g) * std).to(torch.bfloat16))
+    sl = {"x": rnd((rows, w.d), 1.0), "gate": np.full(rows, 1.0 / w.k, np.float32), "Wg": rnd((1, w.d, w.f), 0.02),
+          "Wu": rnd((1, w.d, w.f), 0.02), "Wd": rnd((1, w.f, w.d), 0.02)}
+    if w.backward:
+        sl["dY"] = rnd((rows, w.d), 1.0)
+    for _ in range(args.warmup):
+        oracle_expert_sample(w, [sl], 1, w.backward)
+    secs, flops = 0.0, 0
+    for _ in range(args.steps):
+        s, f, _ = oracle_expert_sample(w, [sl], 1, w.backward)
+        secs += s; flops += f
+    val = flops / secs / 1e12
+    sample = f"{rows} rows of one expert per step ({'fwd+dgrad+wgrad' if w.backward else 'fwd'}), d={w.d}, f={w.f}"
+    print(json.dumps({
+        "impl": "reference", "metric": "moe_layer_tflops", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "T": w.T, "d": w.d, "E": w.E, "k": w.k, "f": w.f},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# --------------------------------------------------------------------------------------- CUDA path
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5_train", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        args.steps = args.steps or 3
+        args.warmup = 1 if args.warmup is None else args.warmup
+        return run_reference(args, w)
+    args.steps = args.steps or 20
+    args.warmup = max(3, args.warmup or 3)
+
+    from paper_2607_01844_b200 import binding
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    inp = synth.make_inputs(w, dev)
+    ctx = binding.context_for(w, device=local, host_io=not args.no_e2e)
+    buf = binding.LayerBuffers(w, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.forward(ctx, inp, buf, stream)
+        if w.backward:
+            binding.backward(ctx, inp, buf, stream)
+
+    for _ in range(args.warmup):
+        step()
+    binding.mop_poll(ctx, stream)
+    binding.mop_profile_enable(ctx, True)
+    sampler = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize()
+    sampler.start()
+    l0 = ctx.launch_count
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize(); barrier()
+    launches = ctx.launch_count - l0
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    prof = binding.mop_profile_read(ctx, stream)
+    binding.mop_profile_enable(ctx, False)
+    binding.mop_poll(ctx, stream)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_step = ms / args.steps
+    value = world * flops_per_step(w) / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        xh = inp["x"].cpu().pin_memory()
+        Yh = torch.empty_like(xh).pin_memory()
+        h2d, d2h = xh.numel() * 2, Yh.numel() * 2
+        if w.backward:
+            dYh = inp["dY"].cpu().pin_memory()
+            dXh = torch.empty_like(xh).pin_memory()
+            dgh = torch.empty((w.T, w.k), dtype=torch.float32).pin_memory()
+            h2d += dYh.numel() * 2
+            d2h += dXh.numel() * 2 + dgh.numel() * 4
+
+            def host_step():
+                binding.mop_moe_train_step_host(ctx, xh, dYh, inp["W_r"], inp["bias"], inp["W_gate"], inp["W_up"],
+                                                inp["W_down"], Yh, dXh, dgh, buf.dW_gate, buf.dW_up, buf.dW_down,
+                                                stream)
+        else:
+            idxh = torch.empty((w.T, w.k), dtype=torch.int32).pin_memory()
+            gh = torch.empty((w.T, w.k), dtype=torch.float32).pin_memory()
+            d2h += idxh.numel() * 4 + gh.numel() * 4
+
+            def host_step():
+                binding.mop_moe_forward_host(ctx, xh, inp["W_r"], inp["bias"], inp["W_gate"], inp["W_up"],
+                                             inp["W_down"], Yh, idxh, gh, stream)
+        for _ in range(2):
+            host_step()
+        n_e2e = min(args.steps, 10)
+        barrier(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n_e2e):
+            host_step()
+        e1.record(stream)
+        torch.cuda.synchronize(); barrier()
+        ems = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ems], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        assert torch.equal(Yh, buf.Y.cpu()), "host entry point and device path disagree"
+        e2e = {"value": world * flops_per_step(w) / (ems / n_e2e * 1e-3) / 1e12, "unit": "TFLOP/s",
+               "ms_per_step": ems / n_e2e, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        return
+    # ---- per-kernel table and the roofline of the dominant kernel
+    pk, pk_kind = peaks()
+    counts = buf.counts.cpu().numpy()
+    work = kernel_work(w, counts)
+    kernels = {}
+    for name, (tot, calls) in prof.items():
+        avg_ms = tot / max(1, calls)
+        fl, by = work.get(name, (0, 0))
+        rec = {"ms": round(avg_ms, 4), "launches": calls, "share": round(tot / ms * (1 if world == 1 else 1), 4)}
+        if fl:
+            rec["tflops"] = round(fl / (avg_ms * 1e-3) / 1e12, 1)
+        if by:
+            rec["gbs"] = round(by / (avg_ms * 1e-3) / 1e9, 1)
+        kernels[name] = rec
+    roofline = None
+    if kernels:
+        top = max(prof, key=lambda n: prof[n][0])
+        avg_s = prof[top][0] / prof[top][1] * 1e-3
+        fl, by = work.get(top, (0, 0))
+        t_tensor = fl / (pk["bf16_tflops_sustained"] * 1e12)
+        t_hbm = by / (pk["hbm_gbs"] * 1e9)
+        if top == "route_score":
+            # plain fp32 FMA chains: 148 SMs x 128 lanes x 2 flop at the maximum SM clock
+            peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            roofline = {"kernel": top, "bound": "alu", "achieved": fl / avg_s / 1e12, "peak": peak, "unit": "TFLOP/s"}
+        elif t_tensor >= t_hbm:
+            roofline = {"kernel": top, "bound": "tensor", "achieved": fl / avg_s / 1e12,
+                        "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+        else:
+            roofline = {"kernel": top, "bound": "hbm", "achieved": by / avg_s / 1e9, "peak": pk["hbm_gbs"],
+                        "unit": "GB/s"}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline["peak_source"] = pk_kind
+        roofline["traffic"] = NCU_TRAFFIC_BYTES.get((top, w.name))
+        roofline["ms"] = avg_s * 1e3
+
+    # ---- CPU baseline: the oracle on a bounded sample (complete work of a few experts)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        order = np.argsort(-counts)
+        mid = [int(e) for e in order[len(order) // 2: len(order) // 2 + 1]]      # a median-load expert
+        sl = expert_slices(w, inp, buf.idx, buf.gate, mid)
+        s1, f1, r1 = oracle_expert_sample(w, sl, 1, w.backward)
+        n = int(max(1, min(16, 15.0 / max(s1, 1e-3))))
+        more = [int(e) for e in order[len(order) // 2 + 1: len(order) // 2 + n]]
+        s2, f2, r2 = oracle_expert_sample(w, expert_slices(w, inp, buf.idx, buf.gate, more), len(more), w.backward)
+        cpu = {"value": (f1 + f2) / (s1 + s2) / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+               "seconds": round(s1 + s2, 2),
+               "sample": f"{1 + len(more)} median-load experts, {r1 + r2} rows: "
+                         f"{'fwd+dgrad+wgrad' if w.backward else 'fwd'} of every row routed to them"}
+
+    out = {
+        "metric": "moe_layer_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "T": w.T, "d": w.d, "E": w.E, "k": w.k, "f": w.f,
+                   "pass": "fwd+bwd" if w.backward else "fwd", "l2": "inputs larger than L2",
+                   "load_cv": float(counts.std() / max(1e-9, counts.mean())),
+                   "empty_experts": int((counts == 0).sum())},
+        "frac_of_bf16_peak_nominal": value / world / 2250.0,
+        "frac_of_bf16_peak_measured": value / world / pk["bf16_tflops_sustained"],
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

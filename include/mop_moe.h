@@ -139,6 +139,27 @@ mop_status mop_moe_forward_host(mop_ctx* ctx, const void* x_host, const float* W
                                 const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
                                 int32_t* idx_host, float* gate_host, void* stream);
 
+/* Whole training step of the layer with HOST activations: copies x and dY in, runs route,
+ * permute, expert_ffn_fwd (keeping G, U), combine and expert_ffn_bwd on `stream`, copies Y, dX
+ * and dgate back, and synchronises.  Weights and weight gradients stay on the device (they are
+ * parameters and optimiser inputs, not step inputs).  Needs with_backward = 1 and host_io = 1.
+ * x_host, dY_host [T,d] bf16; Y_host, dX_host [T,d] bf16 out; dgate_host [T,k] f32 out or NULL;
+ * dW_gate, dW_up [E,d,f], dW_down [E,f,d] f32 DEVICE out. */
+mop_status mop_moe_train_step_host(mop_ctx* ctx, const void* x_host, const void* dY_host, const float* W_r,
+                                   const float* bias, const void* W_gate, const void* W_up, const void* W_down,
+                                   void* Y_host, void* dX_host, float* dgate_host, float* dW_gate, float* dW_up,
+                                   float* dW_down, void* stream);
+
+/* Per-kernel timing.  mop_profile_enable(ctx, 1) creates a pool of CUDA events on first use and
+ * from then on brackets every kernel launch of this context with an event pair on the launching
+ * stream (up to 8192 launches between reads; later ones are not recorded).  mop_profile_read
+ * synchronises `stream`, sums the recorded durations by kernel name into names / total_ms / calls
+ * (arrays of max_names entries; names point to static strings), clears the records and returns
+ * the number of distinct kernels, or -1 on error. */
+mop_status mop_profile_enable(mop_ctx* ctx, int on);
+int32_t mop_profile_read(mop_ctx* ctx, void* stream, int32_t max_names, const char** names, float* total_ms,
+                         int32_t* calls);
+
 #ifdef __cplusplus
 }
 #endif

@@ -58,6 +58,11 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_combine.argtypes = [_P] * 5
         L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 19
         L.mop_moe_forward_host.argtypes = [_P] * 11
+        L.mop_moe_train_step_host.argtypes = [_P] * 15
+        L.mop_profile_enable.argtypes = [_P, ctypes.c_int]
+        L.mop_profile_read.argtypes = [_P, _P, ctypes.c_int32, ctypes.POINTER(ctypes.c_char_p),
+                                       ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
+        L.mop_profile_read.restype = ctypes.c_int32
         _lib = L
     return _lib
 
@@ -153,6 +158,30 @@ def mop_moe_forward_host(ctx, x_host, W_r, bias, W_gate, W_up, W_down, Y_host, i
     _check("mop_moe_forward_host",
            lib().mop_moe_forward_host(ctx.handle, _ptr(x_host), _ptr(W_r), _ptr(bias), _ptr(W_gate), _ptr(W_up),
                                       _ptr(W_down), _ptr(Y_host), _ptr(idx_host), _ptr(gate_host), _stream(stream)))
+
+
+def mop_moe_train_step_host(ctx, x_host, dY_host, W_r, bias, W_gate, W_up, W_down, Y_host, dX_host, dgate_host,
+                            dW_gate, dW_up, dW_down, stream=None):
+    """x_host, dY_host, Y_host, dX_host, dgate_host are HOST tensors; weights and dW are device tensors."""
+    _check("mop_moe_train_step_host",
+           lib().mop_moe_train_step_host(ctx.handle, _ptr(x_host), _ptr(dY_host), _ptr(W_r), _ptr(bias), _ptr(W_gate),
+                                         _ptr(W_up), _ptr(W_down), _ptr(Y_host), _ptr(dX_host), _ptr(dgate_host),
+                                         _ptr(dW_gate), _ptr(dW_up), _ptr(dW_down), _stream(stream)))
+
+
+def mop_profile_enable(ctx, on=True):
+    _check("mop_profile_enable", lib().mop_profile_enable(ctx.handle, int(on)))
+
+
+def mop_profile_read(ctx, stream=None, max_names=64):
+    """{kernel name: (total milliseconds, launches)} since the last read."""
+    names = (ctypes.c_char_p * max_names)()
+    ms = (ctypes.c_float * max_names)()
+    calls = (ctypes.c_int32 * max_names)()
+    n = lib().mop_profile_read(ctx.handle, _stream(stream), max_names, names, ms, calls)
+    if n < 0:
+        raise RuntimeError("mop_profile_read failed")
+    return {names[i].decode(): (float(ms[i]), int(calls[i])) for i in range(n)}
 
 
 class LayerBuffers:

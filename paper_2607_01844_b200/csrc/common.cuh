@@ -27,4 +27,20 @@ __device__ __forceinline__ float sigmoidf_acc(float v) { return 1.0f / (1.0f + e
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Optional per-kernel timing: a pool of CUDA event pairs recorded around every launch on the
+// launching stream, aggregated by kernel name when read.  Off by default (no events, no cost).
+struct Profiler {
+    static constexpr int MAX_REC = 8192;
+    bool on = false;
+    cudaEvent_t* ev = nullptr;          // 2 * MAX_REC events once enabled
+    const char* names[MAX_REC];
+    int n = 0;
+    void begin(const char* name, cudaStream_t st) {
+        if (on && n < MAX_REC) { names[n] = name; cudaEventRecord(ev[2 * n], st); }
+    }
+    void end(cudaStream_t st) {
+        if (on && n < MAX_REC) { cudaEventRecord(ev[2 * n + 1], st); ++n; }
+    }
+};
+
 }  // namespace mop

@@ -500,6 +500,7 @@ struct TcPlan {
     int sm_count;
     mop_moe_shape s;
     void* encode;   // cuTensorMapEncodeTiled
+    Profiler* prof;
 };
 
 struct TcFwdArgs {
@@ -528,8 +529,9 @@ inline mop_status tc_set_smem() {
                                 TC_SMEM_BYTES) == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
-inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count) {
+inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count, Profiler* prof) {
     p->sm_count = sm_count;
+    p->prof = prof;
     p->s = s;
     cudaDriverEntryPointQueryResult q;
     void* fn = nullptr;
@@ -573,9 +575,11 @@ inline bool tc_map_3d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_
 }
 
 template <int KIND>
-inline mop_status tc_launch(const TcPlan* p, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
-                            const CUtensorMap& b1, const TcArgs& args, cudaStream_t st) {
+inline mop_status tc_launch(const TcPlan* p, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                            const CUtensorMap& b0, const CUtensorMap& b1, const TcArgs& args, cudaStream_t st) {
+    p->prof->begin(name, st);
     tc_grouped_gemm_kernel<KIND><<<p->sm_count, TC_THREADS, TC_SMEM_BYTES, st>>>(a0, a1, b0, b1, args);
+    p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
@@ -590,7 +594,9 @@ inline TcArgs tc_base_args(const TcPlan* p, const int32_t* offsets, int32_t* til
 }
 
 inline mop_status tc_build_tiles(const TcPlan* p, const int32_t* offsets, int32_t* tiles, cudaStream_t st) {
+    p->prof->begin("tc_build_mtiles", st);
     tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(offsets, p->s.E, reinterpret_cast<int4*>(tiles + 64), tiles);
+    p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
@@ -610,14 +616,14 @@ inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int3
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
         g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_F1>(p, mXp, mXp, mWg, mWu, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_F1>(p, "gemm_up_swiglu", mXp, mXp, mWg, mWu, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // F2: Yp = gate * (H W_down)
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
         g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_F2>(p, mH, mH, mWd, mWd, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_F2>(p, "gemm_down_gate", mH, mH, mWd, mWd, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     return MOP_OK;
@@ -654,28 +660,28 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
         g.tiles_n = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
         g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
         g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.part = a.part; g.ep.ldo = s.f; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_B2>(p, mdYpA, mdYpA, mWdK, mWdK, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_B2>(p, "gemm_dgrad_down_dswiglu", mdYpA, mdYpA, mWdK, mWdK, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // B4: dXp = dG W_gate^T + dU W_up^T
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
         g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_B4>(p, mdG, mdU, mWgK, mWuK, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_B4>(p, "gemm_dgrad_gate_up", mdG, mdU, mWgK, mWuK, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // WD: dW_down[e] = (gate H)_e^T dYp_e
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.tiles_m_fixed = ceil_div(s.f, TC_BM); g.Mfix = s.f; g.N = s.d;
         g.ep.outf = a.dW_down; g.ep.accumulate = a.accumulate;
-        if ((r = tc_launch<TC_WD>(p, mgH, mgH, mdYpB, mdYpB, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_WD>(p, "gemm_wgrad_down", mgH, mgH, mdYpB, mdYpB, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // WGU: [dW_gate | dW_up][e] = Xp_e^T [dG | dU]_e
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.f, 128); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
         g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate;
-        if ((r = tc_launch<TC_WGU>(p, mXpA, mXpA, mdGB, mdUB, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_WGU>(p, "gemm_wgrad_gate_up", mXpA, mXpA, mdGB, mdUB, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     return MOP_OK;

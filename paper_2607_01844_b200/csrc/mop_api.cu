@@ -32,10 +32,11 @@ struct mop_ctx {
     float* part;         // [ntile_max, M] partial dot products for dgate
     bf16 *dYp, *dG, *dU, *gH, *dXp;  // backward intermediates
     // host-buffer entry point scratch
-    bf16 *hx, *hXp, *hH, *hYp, *hY;
+    bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
     int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
-    float* hgate;
+    float *hgate, *hdgate;
     TcPlan plan;
+    Profiler prof;
 };
 
 namespace {
@@ -45,6 +46,7 @@ inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 struct Layout {
     size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
+    size_t hG, hU, hdY, hdX, hdgate;
     size_t total;
 };
 
@@ -80,6 +82,13 @@ Layout make_layout(const mop_moe_shape& s) {
         L.hperm = take(M * 4);
         L.hsrc = take(M * 4);
         L.hgate = take(M * 4);
+        if (s.with_backward) {
+            L.hG = take(M * f * 2);
+            L.hU = take(M * f * 2);
+            L.hdY = take(T * d * 2);
+            L.hdX = take(T * d * 2);
+            L.hdgate = take(M * 4);
+        }
     }
     L.total = o;
     return L;
@@ -119,6 +128,14 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
         if ((expr) != cudaSuccess) return MOP_ERR_CUDA; \
     } while (0)
 
+// Launch with optional event timing around it.
+#define LAUNCH(c, name, st, ...)       \
+    do {                               \
+        (c)->prof.begin(name, st);     \
+        __VA_ARGS__;                   \
+        (c)->prof.end(st);             \
+    } while (0)
+
 inline mop_status after_launch(mop_ctx* c, int n = 1) {
     c->launches += n;
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
@@ -139,9 +156,9 @@ struct DeviceGuard {
 bool use_tensor(const mop_ctx* c) { return c->tensor_ok && c->s.gemm_path != MOP_GEMM_SCALAR; }
 
 // ---- scalar-path launches ---------------------------------------------------------------
-mop_status launch_scalar(mop_ctx* c, const ScalarGemmArgs& g, cudaStream_t st) {
+mop_status launch_scalar(mop_ctx* c, const char* name, const ScalarGemmArgs& g, cudaStream_t st) {
     dim3 grid(ceil_div(g.N, SG_BN), c->s.E);
-    scalar_grouped_gemm_kernel<<<grid, 256, 0, st>>>(g);
+    LAUNCH(c, name, st, scalar_grouped_gemm_kernel<<<grid, 256, 0, st>>>(g));
     return after_launch(c);
 }
 
@@ -216,10 +233,17 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         c->hperm = reinterpret_cast<int32_t*>(w + L.hperm);
         c->hsrc = reinterpret_cast<int32_t*>(w + L.hsrc);
         c->hgate = reinterpret_cast<float*>(w + L.hgate);
+        if (shape->with_backward) {
+            c->hG = reinterpret_cast<bf16*>(w + L.hG);
+            c->hU = reinterpret_cast<bf16*>(w + L.hU);
+            c->hdY = reinterpret_cast<bf16*>(w + L.hdY);
+            c->hdX = reinterpret_cast<bf16*>(w + L.hdX);
+            c->hdgate = reinterpret_cast<float*>(w + L.hdgate);
+        }
     }
     if (cudaMemset(c->status, 0, 256) != cudaSuccess) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
     if (c->tensor_ok) {
-        st = tc_plan_init(&c->plan, *shape, c->sm_count);
+        st = tc_plan_init(&c->plan, *shape, c->sm_count, &c->prof);
         if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
     }
     *out = c;
@@ -229,6 +253,10 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
 void mop_destroy(mop_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
+    if (c->prof.ev) {
+        for (int i = 0; i < 2 * Profiler::MAX_REC; ++i) cudaEventDestroy(c->prof.ev[i]);
+        delete[] c->prof.ev;
+    }
     cudaFree(c->ws);
     delete c;
 }
@@ -264,12 +292,14 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* z = logits_opt ? logits_opt : c->z;
     dim3 grid(ceil_div(s.T, SC_TT), ceil_div(s.E, SC_TE));
-    route_score_kernel<<<grid, 256, 0, st>>>(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E);
+    LAUNCH(c, "route_score", st,
+           route_score_kernel<<<grid, 256, 0, st>>>(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E));
     mop_status r = after_launch(c);
     if (r != MOP_OK) return r;
     const size_t smem = (size_t)SEL_WARPS * 2 * s.E * sizeof(float);
-    route_select_kernel<<<ceil_div(s.T, SEL_WARPS), SEL_WARPS * 32, smem, st>>>(z, bias, topk_idx, topk_gate, s.T, s.E,
-                                                                               s.k, s.score_fn, s.bias_mode);
+    LAUNCH(c, "route_select", st,
+           route_select_kernel<<<ceil_div(s.T, SEL_WARPS), SEL_WARPS * 32, smem, st>>>(
+               z, bias, topk_idx, topk_gate, s.T, s.E, s.k, s.score_fn, s.bias_mode));
     return after_launch(c);
 }
 
@@ -287,18 +317,23 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
     const size_t smem = (size_t)PERM_WARPS * s.E * sizeof(int32_t);
     mop_status r;
     if (units > 0) {
-        perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, M, s.E);
+        LAUNCH(c, "perm_hist", st,
+               perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, M,
+                                                                                            s.E));
         if ((r = after_launch(c)) != MOP_OK) return r;
     }
-    perm_scan_kernel<<<1, 1024, (s.E + 1) * sizeof(int32_t), st>>>(c->partial, counts, offsets, units, s.E);
+    LAUNCH(c, "perm_scan", st,
+           perm_scan_kernel<<<1, 1024, (s.E + 1) * sizeof(int32_t), st>>>(c->partial, counts, offsets, units, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
     if (units == 0) return MOP_OK;
-    perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, perm_row,
-                                                                                row_src, M, s.E);
+    LAUNCH(c, "perm_rank", st,
+           perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, perm_row,
+                                                                                        row_src, M, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
     const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
-    scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, s.T,
-                                                s.k, s.d / 8);
+    LAUNCH(c, "permute_scatter_rows", st,
+           scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row,
+                                                       s.T, s.k, s.d / 8));
     return after_launch(c);
 }
 
@@ -310,8 +345,10 @@ mop_status mop_moe_combine(mop_ctx* c, const void* Yp, const int32_t* perm_row, 
     DeviceGuard guard(c->device);
     if (!guard.ok) return MOP_ERR_CUDA;
     const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
-    combine_rows_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint4*>(Yp), perm_row, static_cast<uint4*>(Y), s.T, s.k, s.d / 8);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    LAUNCH(c, "combine_rows", st,
+           combine_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(Yp), perm_row, static_cast<uint4*>(Y),
+                                                       s.T, s.k, s.d / 8));
     return after_launch(c);
 }
 
@@ -348,14 +385,14 @@ mop_status mop_moe_expert_ffn_fwd(mop_ctx* c, const void* Xp, const int32_t* off
     g.offsets = offsets; g.ragged_k = 0; g.N = s.f; g.Kfix = s.d; g.npairs = 2; g.dual_acc = 1; g.epi = EPI_SWIGLU;
     g.ep.out0 = static_cast<bf16*>(H); g.ep.out1 = static_cast<bf16*>(G_save); g.ep.out2 = static_cast<bf16*>(U_save);
     g.ep.ldo = s.f; g.ep.M_total = M;
-    mop_status r = launch_scalar(c, g, st);
+    mop_status r = launch_scalar(c, "scalar_up_swiglu", g, st);
     if (r != MOP_OK) return r;
     ScalarGemmArgs h{};
     h.A[0] = static_cast<const bf16*>(H); h.B[0] = static_cast<const bf16*>(W_down);
     h.sAm = s.f; h.sAk = 1; h.sBk = s.d; h.sBn = 1; h.sBe = (long)s.d * s.f;
     h.offsets = offsets; h.ragged_k = 0; h.N = s.d; h.Kfix = s.f; h.npairs = 1; h.epi = EPI_GATE;
     h.ep.out0 = static_cast<bf16*>(Yp); h.ep.gate = topk_gate; h.ep.row_src = row_src; h.ep.ldo = s.d; h.ep.M_total = M;
-    return launch_scalar(c, h, st);
+    return launch_scalar(c, "scalar_down_gate", h, st);
 }
 
 mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, const void* G_save,
@@ -377,8 +414,10 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
     if (s.T > 0) {
         // dYp[p,:] = dY[t,:]  (unscaled; the gate enters through dH and gate*H)
         const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
-        scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dY), reinterpret_cast<uint4*>(c->dYp),
-                                                    perm_row, s.T, s.k, s.d / 8);
+        LAUNCH(c, "dy_scatter_rows", st,
+               scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dY),
+                                                           reinterpret_cast<uint4*>(c->dYp), perm_row, s.T, s.k,
+                                                           s.d / 8));
         if ((r = after_launch(c)) != MOP_OK) return r;
     }
     int ntile_part = 0;
@@ -405,7 +444,7 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
             g.ep.in0 = static_cast<const bf16*>(G_save); g.ep.in1 = static_cast<const bf16*>(U_save);
             g.ep.in2 = static_cast<const bf16*>(H);
             g.ep.gate = topk_gate; g.ep.row_src = row_src; g.ep.part = c->part; g.ep.ldo = s.f; g.ep.M_total = M;
-            if ((r = launch_scalar(c, g, st)) != MOP_OK) return r;
+            if ((r = launch_scalar(c, "scalar_dgrad_down", g, st)) != MOP_OK) return r;
             ntile_part = ceil_div(s.f, SG_BN);
             ScalarGemmArgs h{};  // dXp = dG W_gate^T + dU W_up^T
             h.A[0] = c->dG; h.A[1] = c->dU;
@@ -413,50 +452,128 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
             h.sAm = s.f; h.sAk = 1; h.sBk = 1; h.sBn = s.f; h.sBe = (long)s.d * s.f;
             h.offsets = offsets; h.N = s.d; h.Kfix = s.f; h.npairs = 2; h.dual_acc = 0; h.epi = EPI_BF16;
             h.ep.out0 = c->dXp; h.ep.ldo = s.d; h.ep.M_total = M;
-            if ((r = launch_scalar(c, h, st)) != MOP_OK) return r;
+            if ((r = launch_scalar(c, "scalar_dgrad_gate_up", h, st)) != MOP_OK) return r;
         }
         // weight gradients (ragged K = the expert's rows); run even for T = 0 so that dW is defined
         ScalarGemmArgs w{};
         w.offsets = offsets; w.ragged_k = 1; w.npairs = 1; w.epi = EPI_F32; w.ep.accumulate = s.dw_accumulate;
         w.A[0] = c->gH; w.sAm = 1; w.sAk = s.f; w.B[0] = c->dYp; w.sBk = s.d; w.sBn = 1;
         w.Mfix = s.f; w.N = s.d; w.ep.outf = dW_down;
-        if ((r = launch_scalar(c, w, st)) != MOP_OK) return r;
+        if ((r = launch_scalar(c, "scalar_wgrad", w, st)) != MOP_OK) return r;
         w.A[0] = static_cast<const bf16*>(Xp); w.sAm = 1; w.sAk = s.d; w.B[0] = c->dG; w.sBk = s.f; w.sBn = 1;
         w.Mfix = s.d; w.N = s.f; w.ep.outf = dW_gate;
-        if ((r = launch_scalar(c, w, st)) != MOP_OK) return r;
+        if ((r = launch_scalar(c, "scalar_wgrad", w, st)) != MOP_OK) return r;
         w.B[0] = c->dU; w.ep.outf = dW_up;
-        if ((r = launch_scalar(c, w, st)) != MOP_OK) return r;
+        if ((r = launch_scalar(c, "scalar_wgrad", w, st)) != MOP_OK) return r;
     }
     if (s.T == 0) return MOP_OK;
-    dgate_reduce_kernel<<<ceil_div(M, 256), 256, 0, st>>>(c->part, perm_row, dgate, M, ntile_part);
+    LAUNCH(c, "dgate_reduce", st,
+           dgate_reduce_kernel<<<ceil_div(M, 256), 256, 0, st>>>(c->part, perm_row, dgate, M, ntile_part));
     if ((r = after_launch(c)) != MOP_OK) return r;
     return mop_moe_combine(c, c->dXp, perm_row, dX, stream);
 }
 
-mop_status mop_moe_forward_host(mop_ctx* c, const void* x_host, const float* W_r, const float* bias,
-                                const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
-                                int32_t* idx_host, float* gate_host, void* stream) {
-    if (!c || !x_host || !Y_host) return MOP_ERR_INVALID_ARG;
-    if (!c->s.host_io) return MOP_ERR_UNSUPPORTED;
+namespace {
+mop_status step_host(mop_ctx* c, const void* x_host, const void* dY_host, const float* W_r, const float* bias,
+                     const void* W_gate, const void* W_up, const void* W_down, void* Y_host, int32_t* idx_host,
+                     float* gate_host, void* dX_host, float* dgate_host, float* dW_gate, float* dW_up, float* dW_down,
+                     void* stream) {
     const mop_moe_shape& s = c->s;
+    const bool bwd = dY_host != nullptr;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MOP_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t M = (size_t)s.T * s.k;
-    CUDA_OK(cudaMemcpyAsync(c->hx, x_host, (size_t)s.T * s.d * 2, cudaMemcpyHostToDevice, st));
+    const size_t M = (size_t)s.T * s.k, xb = (size_t)s.T * s.d * 2;
+    if (s.T > 0) {
+        CUDA_OK(cudaMemcpyAsync(c->hx, x_host, xb, cudaMemcpyHostToDevice, st));
+        if (bwd) CUDA_OK(cudaMemcpyAsync(c->hdY, dY_host, xb, cudaMemcpyHostToDevice, st));
+    }
     mop_status r;
     if ((r = mop_moe_route(c, c->hx, W_r, bias, c->hidx, c->hgate, nullptr, stream)) != MOP_OK) return r;
     if ((r = mop_moe_permute(c, c->hx, c->hidx, c->hcounts, c->hoffsets, c->hperm, c->hsrc, c->hXp, stream)) != MOP_OK)
         return r;
-    if ((r = mop_moe_expert_ffn_fwd(c, c->hXp, c->hoffsets, c->hsrc, c->hgate, W_gate, W_up, W_down, nullptr, nullptr,
-                                    c->hH, c->hYp, stream)) != MOP_OK)
+    if ((r = mop_moe_expert_ffn_fwd(c, c->hXp, c->hoffsets, c->hsrc, c->hgate, W_gate, W_up, W_down,
+                                    bwd ? c->hG : nullptr, bwd ? c->hU : nullptr, c->hH, c->hYp, stream)) != MOP_OK)
         return r;
     if ((r = mop_moe_combine(c, c->hYp, c->hperm, c->hY, stream)) != MOP_OK) return r;
-    CUDA_OK(cudaMemcpyAsync(Y_host, c->hY, (size_t)s.T * s.d * 2, cudaMemcpyDeviceToHost, st));
-    if (idx_host) CUDA_OK(cudaMemcpyAsync(idx_host, c->hidx, M * 4, cudaMemcpyDeviceToHost, st));
-    if (gate_host) CUDA_OK(cudaMemcpyAsync(gate_host, c->hgate, M * 4, cudaMemcpyDeviceToHost, st));
+    if (bwd) {
+        if ((r = mop_moe_expert_ffn_bwd(c, c->hdY, c->hXp, c->hG, c->hU, c->hH, c->hoffsets, c->hperm, c->hsrc,
+                                        c->hgate, W_gate, W_up, W_down, c->hdX, dW_gate, dW_up, dW_down, c->hdgate,
+                                        stream)) != MOP_OK)
+            return r;
+    }
+    if (s.T > 0) {
+        CUDA_OK(cudaMemcpyAsync(Y_host, c->hY, xb, cudaMemcpyDeviceToHost, st));
+        if (idx_host) CUDA_OK(cudaMemcpyAsync(idx_host, c->hidx, M * 4, cudaMemcpyDeviceToHost, st));
+        if (gate_host) CUDA_OK(cudaMemcpyAsync(gate_host, c->hgate, M * 4, cudaMemcpyDeviceToHost, st));
+        if (bwd) {
+            CUDA_OK(cudaMemcpyAsync(dX_host, c->hdX, xb, cudaMemcpyDeviceToHost, st));
+            if (dgate_host) CUDA_OK(cudaMemcpyAsync(dgate_host, c->hdgate, M * 4, cudaMemcpyDeviceToHost, st));
+        }
+    }
     CUDA_OK(cudaStreamSynchronize(st));
     return MOP_OK;
+}
+}  // namespace
+
+mop_status mop_moe_forward_host(mop_ctx* c, const void* x_host, const float* W_r, const float* bias,
+                                const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
+                                int32_t* idx_host, float* gate_host, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (c->s.T > 0 && (!x_host || !Y_host)) return MOP_ERR_INVALID_ARG;
+    if (!c->s.host_io) return MOP_ERR_UNSUPPORTED;
+    return step_host(c, x_host, nullptr, W_r, bias, W_gate, W_up, W_down, Y_host, idx_host, gate_host, nullptr,
+                     nullptr, nullptr, nullptr, nullptr, stream);
+}
+
+mop_status mop_moe_train_step_host(mop_ctx* c, const void* x_host, const void* dY_host, const float* W_r,
+                                   const float* bias, const void* W_gate, const void* W_up, const void* W_down,
+                                   void* Y_host, void* dX_host, float* dgate_host, float* dW_gate, float* dW_up,
+                                   float* dW_down, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (c->s.T > 0 && (!x_host || !dY_host || !Y_host || !dX_host)) return MOP_ERR_INVALID_ARG;
+    if (!c->s.host_io || !c->s.with_backward) return MOP_ERR_UNSUPPORTED;
+    if (c->s.T == 0 && !dY_host) dY_host = c;  // any non-null token: selects the backward branch
+    return step_host(c, x_host, dY_host, W_r, bias, W_gate, W_up, W_down, Y_host, nullptr, nullptr, dX_host,
+                     dgate_host, dW_gate, dW_up, dW_down, stream);
+}
+
+mop_status mop_profile_enable(mop_ctx* c, int on) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    if (on && !c->prof.ev) {
+        c->prof.ev = new (std::nothrow) cudaEvent_t[2 * Profiler::MAX_REC];
+        if (!c->prof.ev) return MOP_ERR_WORKSPACE;
+        for (int i = 0; i < 2 * Profiler::MAX_REC; ++i)
+            if (cudaEventCreate(&c->prof.ev[i]) != cudaSuccess) return MOP_ERR_CUDA;
+    }
+    c->prof.on = on != 0;
+    c->prof.n = 0;
+    return MOP_OK;
+}
+
+int32_t mop_profile_read(mop_ctx* c, void* stream, int32_t max_names, const char** names, float* total_ms,
+                         int32_t* calls) {
+    if (!c || !names || !total_ms || !calls || max_names < 1) return -1;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return -1;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return -1;
+    int32_t n = 0;
+    for (int i = 0; i < c->prof.n; ++i) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, c->prof.ev[2 * i], c->prof.ev[2 * i + 1]) != cudaSuccess) return -1;
+        int32_t j = 0;
+        while (j < n && names[j] != c->prof.names[i]) ++j;   // names are string literals: compare pointers
+        if (j == n) {
+            if (n == max_names) continue;
+            names[n] = c->prof.names[i]; total_ms[n] = 0.0f; calls[n] = 0; ++n;
+        }
+        total_ms[j] += ms;
+        calls[j] += 1;
+    }
+    c->prof.n = 0;
+    return n;
 }
 
 }  // extern "C"
