@@ -204,10 +204,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5_train", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--shape", default=None,
+                    help="T,d,E,k,f overriding the named workload's sizes (same distributions): small cases for "
+                         "profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
+    if args.shape:
+        T, d, E, k, f = (int(v) for v in args.shape.split(","))
+        import dataclasses
+        w = dataclasses.replace(w, T=T, d=d, E=E, k=k, f=f, name=f"{w.name}[{args.shape}]")
     if args.impl == "reference":
         args.steps = args.steps or 3
         args.warmup = 1 if args.warmup is None else args.warmup

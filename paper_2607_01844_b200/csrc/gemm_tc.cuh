@@ -25,13 +25,12 @@ namespace mop {
 
 enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5 };
 
-constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64, TC_STAGES = 4;
+constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // 16 KiB
 constexpr int TC_B_BYTES = TC_BN * TC_BK * 2;   // 32 KiB
 constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 constexpr int TC_CHUNK_BYTES = 64 * TC_BK * 2;  // one 64-wide MN chunk of 64 K rows: 8 KiB
-constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
-constexpr int TC_THREADS = 192;
+constexpr int TC_BAR_BYTES = 1024;                // barriers, TMEM slot, abort flag (keeps 1 KiB alignment)
 constexpr long long TC_WAIT_CYCLES = 4000000000ll;  // about two seconds
 
 template <int KIND>
@@ -43,6 +42,13 @@ struct TcTraits {
     static constexpr bool B_WEIGHT = !RAGGED_K;                       // B is an [E, ., .] weight tensor
     static constexpr int PHASES = (KIND == TC_B4) ? 2 : 1;
     static constexpr int N_PER_TILE = DUAL_B ? 128 : 256;             // output columns per tensor per tile
+    // Weight gradients have a short K loop (the expert's rows) and a 128 KiB fp32 tile to write, so
+    // they run eight epilogue warps (two per TMEM lane quarter, 128 columns each).
+    static constexpr int STAGES = 4;
+    static constexpr int EPI_WARPS = RAGGED_K ? 8 : 4;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    static constexpr int STORE_BYTES = RAGGED_K ? EPI_WARPS * 4096 : 0;   // 32x32 fp32 transpose buffer per warp
+    static constexpr int SMEM_BYTES = STAGES * TC_STAGE_BYTES + 1024 /*align*/ + TC_BAR_BYTES + STORE_BYTES;
 };
 
 struct TcArgs {
@@ -121,6 +127,25 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         "[%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+// shared -> global tile store (or fp32 add) of one box; completion is tracked by bulk groups
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map),
+                 "r"(src), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                     map),
+                 "r"(src), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -166,6 +191,30 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Same load without the wait, so that several can be in flight; tmem_ld_wait then orders every
+// later use of the destination registers after the wait.
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait(float (&a)[32], float (&b)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    // empty statements that "modify" the registers: nothing that reads them can move above the wait
+#pragma unroll
+    for (int i = 0; i < 32; ++i) asm volatile("" : "+f"(a[i]), "+f"(b[i]));
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (Blackwell).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
@@ -200,11 +249,11 @@ __device__ __forceinline__ TileInfo decode_tile(const TcArgs& a, int t) {
         const int r = t - ti.e * per_e;
         ti.m0 = (r / a.tiles_n) * TC_BM;
         ti.nt = r % a.tiles_n;
-        ti.row0 = a.offsets[ti.e];
-        ti.rows = a.offsets[ti.e + 1] - ti.row0;
+        ti.row0 = __ldg(a.offsets + ti.e);
+        ti.rows = __ldg(a.offsets + ti.e + 1) - ti.row0;
         ti.skip = ti.rows <= 0;
     } else {
-        const int4 m = a.mtiles[t / a.tiles_n];
+        const int4 m = __ldg(a.mtiles + t / a.tiles_n);
         ti.e = m.x; ti.row0 = m.y; ti.rows = m.z; ti.m0 = 0;
         ti.nt = t % a.tiles_n;
         ti.skip = false;
@@ -237,11 +286,13 @@ __global__ void __launch_bounds__(1024) tc_build_mtiles_kernel(const int32_t* __
 
 // ------------------------------------------------------------------------------------------ kernel
 template <int KIND>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TcTraits<KIND>::THREADS, 1)
 tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                        const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
+                       const __grid_constant__ CUtensorMap tmO0, const __grid_constant__ CUtensorMap tmO1,
                        const TcArgs args) {
     using Tr = TcTraits<KIND>;
+    constexpr int TC_STAGES = Tr::STAGES;
     extern __shared__ uint8_t tc_smem_raw[];
     // 1024-byte alignment: the swizzle pattern is a function of address bits 7..9
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -260,7 +311,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), Tr::EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB0);
@@ -281,8 +332,11 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         // ===================================================================== TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool alive = true;
+            // the next tile's descriptor is fetched one tile ahead so that its latency is hidden
+            TileInfo nxt = decode_tile<KIND>(args, min((int)blockIdx.x, max(total_tiles - 1, 0)));
             for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
-                const TileInfo ti = decode_tile<KIND>(args, t);
+                const TileInfo ti = nxt;
+                if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
                 if (ti.skip) continue;
                 const int n0 = ti.nt * Tr::N_PER_TILE;
                 const int nkb = Tr::RAGGED_K ? (ti.rows + TC_BK - 1) / TC_BK : Tr::PHASES * args.kblocks;
@@ -325,8 +379,10 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         // 8 K rows are 1024 bytes apart (stride offset); K-major: 8-row groups 1024 bytes apart.
         constexpr uint32_t mn_lbo = TC_CHUNK_BYTES, mn_sbo = 1024u;
         int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
+        TileInfo nxt = decode_tile<KIND>(args, min((int)blockIdx.x, max(total_tiles - 1, 0)));
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
-            const TileInfo ti = decode_tile<KIND>(args, t);
+            const TileInfo ti = nxt;
+            if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
             if (ti.skip) continue;
             const int buf = it & 1;
             const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
@@ -342,16 +398,16 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
                 const uint32_t sB = sA + TC_A_BYTES;
                 if constexpr (Tr::RAGGED_K) {
-                    // K tail: rows past the expert's end belong to the next expert -> zero them
+                    // K tail: rows past the expert's end belong to the next expert.  Zeroing them in
+                    // the A operand alone makes their products vanish (inputs are finite).
                     const int valid = ti.rows - kb * TC_BK;
                     if (valid < TC_BK) {
                         uint8_t* base = smem + stage * TC_STAGE_BYTES;
-                        const int nrows = TC_BK - valid;
-                        for (int i = lane; i < 6 * nrows * 8; i += 32) {
-                            const int chunk = i / (nrows * 8), rem = i % (nrows * 8);
-                            const int row = valid + rem / 8, v = rem % 8;
-                            *reinterpret_cast<uint4*>(base + chunk * TC_CHUNK_BYTES + row * 128 + v * 16) =
-                                make_uint4(0, 0, 0, 0);
+                        const int n16 = (TC_BK - valid) * 8;     // 16-byte vectors per chunk to clear
+                        for (int i = lane; i < n16; i += 32) {
+                            const int off = (valid + (i >> 3)) * 128 + (i & 7) * 16;
+                            *reinterpret_cast<uint4*>(base + off) = make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4*>(base + TC_CHUNK_BYTES + off) = make_uint4(0, 0, 0, 0);
                         }
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
@@ -380,14 +436,17 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         // ===================================================================== epilogue (4 warps)
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 belong to this warp
         const int r = quarter * 32 + lane;       // row of the tile owned by this thread
+        const int half = (warp - 2) >> 2;        // eight-warp epilogue: columns [128*half, 128*half + 128)
         int it = 0;
+        TileInfo nxt = decode_tile<KIND>(args, min((int)blockIdx.x, max(total_tiles - 1, 0)));
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-            const TileInfo ti = decode_tile<KIND>(args, t);
+            const TileInfo ti = nxt;
+            if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
             const int n0 = ti.nt * Tr::N_PER_TILE;
             if constexpr (Tr::RAGGED_K) {
                 if (ti.skip) {
                     // expert without rows: its gradient is zero (or unchanged when accumulating)
-                    if (!args.ep.accumulate && ti.m0 + r < args.Mfix) {
+                    if (!args.ep.accumulate && half == 0 && ti.m0 + r < args.Mfix) {
                         const size_t ro = ((size_t)ti.e * args.Mfix + ti.m0 + r) * args.N;
                         for (int c = 0; c < TC_BN; c += 4) {
                             const int cc = Tr::DUAL_B ? (c & 127) : c;
@@ -456,19 +515,44 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                     }
                 }
             } else {
-                const size_t ro = ((size_t)ti.e * args.Mfix + ti.m0 + r) * args.N;
+                // Weight-gradient tile: each warp transposes 32 rows x 32 fp32 columns through shared
+                // memory (128-byte rows, 16-byte chunks XOR-swizzled by row: conflict-free both ways)
+                // so that its global stores are whole 128-byte lines: 8 lanes per row, 4 rows per
+                // instruction.  Rows >= Mfix and columns >= N are not written.
+                float* sb = reinterpret_cast<float*>(smem + TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + (warp - 2) * 4096);
+                float* outp = (Tr::DUAL_B && half) ? args.outf1 : args.ep.outf;
+                const int row_base = ti.m0 + quarter * 32;
+                const size_t obase = ((size_t)ti.e * args.Mfix + row_base) * args.N;
+                float acc_b[32];
 #pragma unroll 1
-                for (int c = 0; c < TC_BN; c += 32) {
-                    tmem_ld32(taddr + c, acc);
-                    const int cc = Tr::DUAL_B ? (c & 127) : c;
-                    float* dst = (Tr::DUAL_B && c >= 128) ? args.outf1 : args.ep.outf;
-                    if (row_ok && n0 + cc < args.N) {
+                for (int c = half * 128; c < half * 128 + 128; c += 64) {
+                    tmem_ld32_nowait(taddr + c, acc);
+                    tmem_ld32_nowait(taddr + c + 32, acc_b);
+                    tmem_ld_wait(acc, acc_b);
 #pragma unroll
-                        for (int s = 0; s < 32; s += 8) {
-                            float a8[8];
+                    for (int h = 0; h < 2; ++h) {
+                        __syncwarp();
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
-                            epi_f32<8>(dst + ro + n0 + cc + s, a8, args.ep.accumulate);
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 v = h ? make_float4(acc_b[4 * j], acc_b[4 * j + 1], acc_b[4 * j + 2], acc_b[4 * j + 3])
+                                               : make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+                            *reinterpret_cast<float4*>(sb + lane * 32 + ((j ^ (lane & 7)) << 2)) = v;
+                        }
+                        __syncwarp();
+                        const int col = c + 32 * h;
+                        const int gcol = n0 + (Tr::DUAL_B ? (col & 127) : col) + (lane & 7) * 4;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int rr = 4 * i + (lane >> 3);
+                            float4 v = *reinterpret_cast<const float4*>(sb + rr * 32 + (((lane & 7) ^ (rr & 7)) << 2));
+                            if (row_base + rr < args.Mfix && gcol < args.N) {
+                                float4* dst = reinterpret_cast<float4*>(outp + obase + (size_t)rr * args.N + gcol);
+                                if (args.ep.accumulate) {
+                                    const float4 o = *dst;
+                                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                                }
+                                *dst = v;
+                            }
                         }
                     }
                 }
@@ -526,7 +610,8 @@ typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, 
 template <int KIND>
 inline mop_status tc_set_smem() {
     return cudaFuncSetAttribute(tc_grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                TC_SMEM_BYTES) == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+                                TcTraits<KIND>::SMEM_BYTES) == cudaSuccess
+               ? MOP_OK : MOP_ERR_CUDA;
 }
 
 inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count, Profiler* prof) {
@@ -574,11 +659,26 @@ inline bool tc_map_3d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_
                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D map over a dense [E, rows, cols] fp32 tensor for stores; box = {32 cols, 32 rows, 1}.
+inline bool tc_map_out_f32(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows,
+                           uint64_t cols) {
+    const cuuint64_t dims[3] = {cols, rows, E};
+    const cuuint64_t strides[2] = {cols * 4, rows * cols * 4};
+    const cuuint32_t box[3] = {32, 32, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int KIND>
 inline mop_status tc_launch(const TcPlan* p, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
-                            const CUtensorMap& b0, const CUtensorMap& b1, const TcArgs& args, cudaStream_t st) {
+                            const CUtensorMap& b0, const CUtensorMap& b1, const CUtensorMap& o0, const CUtensorMap& o1,
+                            const TcArgs& args, cudaStream_t st) {
     p->prof->begin(name, st);
-    tc_grouped_gemm_kernel<KIND><<<p->sm_count, TC_THREADS, TC_SMEM_BYTES, st>>>(a0, a1, b0, b1, args);
+    tc_grouped_gemm_kernel<KIND><<<p->sm_count, TcTraits<KIND>::THREADS, TcTraits<KIND>::SMEM_BYTES, st>>>(
+        a0, a1, b0, b1, o0, o1, args);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
@@ -616,14 +716,14 @@ inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int3
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
         g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_F1>(p, "gemm_up_swiglu", mXp, mXp, mWg, mWu, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_F1>(p, "gemm_up_swiglu", mXp, mXp, mWg, mWu, mXp, mXp, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // F2: Yp = gate * (H W_down)
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
         g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_F2>(p, "gemm_down_gate", mH, mH, mWd, mWd, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_F2>(p, "gemm_down_gate", mH, mH, mWd, mWd, mH, mH, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     return MOP_OK;
@@ -647,7 +747,10 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
     mop_status r;
     if ((r = tc_build_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
     ++*launches;
-    CUtensorMap mdYpA, mWdK, mdG, mdU, mWgK, mWuK, mgH, mdYpB, mXpA, mdGB, mdUB;
+    CUtensorMap mdYpA, mWdK, mdG, mdU, mWgK, mWuK, mgH, mdYpB, mXpA, mdGB, mdUB, moWd, moWg, moWu;
+    if (!tc_map_out_f32(p, &moWd, a.dW_down, s.E, s.f, s.d) || !tc_map_out_f32(p, &moWg, a.dW_gate, s.E, s.d, s.f) ||
+        !tc_map_out_f32(p, &moWu, a.dW_up, s.E, s.d, s.f))
+        return MOP_ERR_CUDA;
     if (!tc_map_2d(p, &mdYpA, a.dYp, M, s.d, 128) || !tc_map_3d(p, &mWdK, a.W_down, s.E, s.f, s.d, 256) ||
         !tc_map_2d(p, &mdG, a.dG, M, s.f, 128) || !tc_map_2d(p, &mdU, a.dU, M, s.f, 128) ||
         !tc_map_3d(p, &mWgK, a.W_gate, s.E, s.d, s.f, 256) || !tc_map_3d(p, &mWuK, a.W_up, s.E, s.d, s.f, 256) ||
@@ -660,28 +763,28 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
         g.tiles_n = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
         g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
         g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.part = a.part; g.ep.ldo = s.f; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_B2>(p, "gemm_dgrad_down_dswiglu", mdYpA, mdYpA, mWdK, mWdK, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_B2>(p, "gemm_dgrad_down_dswiglu", mdYpA, mdYpA, mWdK, mWdK, mdYpA, mdYpA, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // B4: dXp = dG W_gate^T + dU W_up^T
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
         g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_B4>(p, "gemm_dgrad_gate_up", mdG, mdU, mWgK, mWuK, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_B4>(p, "gemm_dgrad_gate_up", mdG, mdU, mWgK, mWuK, mdG, mdG, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // WD: dW_down[e] = (gate H)_e^T dYp_e
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.tiles_m_fixed = ceil_div(s.f, TC_BM); g.Mfix = s.f; g.N = s.d;
         g.ep.outf = a.dW_down; g.ep.accumulate = a.accumulate;
-        if ((r = tc_launch<TC_WD>(p, "gemm_wgrad_down", mgH, mgH, mdYpB, mdYpB, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_WD>(p, "gemm_wgrad_down", mgH, mgH, mdYpB, mdYpB, moWd, moWd, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // WGU: [dW_gate | dW_up][e] = Xp_e^T [dG | dU]_e
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.f, 128); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
         g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate;
-        if ((r = tc_launch<TC_WGU>(p, "gemm_wgrad_gate_up", mXpA, mXpA, mdGB, mdUB, g, st)) != MOP_OK) return r;
+        if ((r = tc_launch<TC_WGU>(p, "gemm_wgrad_gate_up", mXpA, mXpA, mdGB, mdUB, moWg, moWu, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     return MOP_OK;
