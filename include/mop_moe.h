@@ -160,6 +160,26 @@ mop_status mop_profile_enable(mop_ctx* ctx, int on);
 int32_t mop_profile_read(mop_ctx* ctx, void* stream, int32_t max_names, const char** names, float* total_ms,
                          int32_t* calls);
 
+/* The same permutation as mop_moe_permute for callers that may not allocate device memory (the
+ * paper has no counterpart; this is a property of the library, not of the method).  A process
+ * that gave all of HBM to its own arena, or a loop that cannot take the device-wide
+ * synchronisation of an allocation, cannot create a context (mop_create calls cudaMalloc).  This
+ * entry point needs none: its only scratch, the per-segment expert histogram, is a 1 MiB array
+ * compiled into the library, resident on every GPU that loads it until the process exits.
+ *   - Limit: ceil(T*k / 512) * E <= 262144, otherwise MOP_ERR_SHAPE and nothing is launched
+ *     (for example T*k = 131072 with E up to 1024).  Also E <= 1024, k <= 32, d % 8 == 0.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on a device
+ *     looks up the array's device address (cudaGetSymbolAddress) and the SM count; make that
+ *     first call outside any stream capture.
+ *   - Every call on a device uses the same array and leaves its last contents there.  Nothing has
+ *     to be cleared between calls (each call overwrites every entry it reads), but two calls
+ *     that overlap on the GPU, on different streams or from different threads, race on it:
+ *     serialise them.
+ * Arguments as in mop_moe_permute, with the shape passed directly and `device` the CUDA ordinal. */
+mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, int32_t k, const void* x,
+                                  const int32_t* topk_idx, int32_t* counts, int32_t* offsets, int32_t* perm_row,
+                                  int32_t* row_src, void* Xp, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 19
         L.mop_moe_forward_host.argtypes = [_P] * 11
         L.mop_moe_train_step_host.argtypes = [_P] * 15
+        L.mop_moe_permute_static.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 4 + [_P] * 8
         L.mop_profile_enable.argtypes = [_P, ctypes.c_int]
         L.mop_profile_read.argtypes = [_P, _P, ctypes.c_int32, ctypes.POINTER(ctypes.c_char_p),
                                        ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
@@ -167,6 +168,13 @@ def mop_moe_train_step_host(ctx, x_host, dY_host, W_r, bias, W_gate, W_up, W_dow
            lib().mop_moe_train_step_host(ctx.handle, _ptr(x_host), _ptr(dY_host), _ptr(W_r), _ptr(bias), _ptr(W_gate),
                                          _ptr(W_up), _ptr(W_down), _ptr(Y_host), _ptr(dX_host), _ptr(dgate_host),
                                          _ptr(dW_gate), _ptr(dW_up), _ptr(dW_down), _stream(stream)))
+
+
+def mop_moe_permute_static(device, T, d, E, k, x, topk_idx, counts, offsets, perm_row, row_src, Xp, stream=None):
+    """Permutation for callers that may not allocate: no context, scratch compiled into the library."""
+    _check("mop_moe_permute_static",
+           lib().mop_moe_permute_static(device, T, d, E, k, _ptr(x), _ptr(topk_idx), _ptr(counts), _ptr(offsets),
+                                        _ptr(perm_row), _ptr(row_src), _ptr(Xp), _stream(stream)))
 
 
 def mop_profile_enable(ctx, on=True):

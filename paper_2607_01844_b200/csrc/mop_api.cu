@@ -5,6 +5,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <mutex>
 #include <new>
 
 #include "common.cuh"
@@ -574,6 +575,81 @@ int32_t mop_profile_read(mop_ctx* c, void* stream, int32_t max_names, const char
     }
     c->prof.n = 0;
     return n;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Permutation without any allocation.  Some callers may not call cudaMalloc at all: a serving
+// or training process that handed the whole HBM to its own arena at start-up (a second
+// allocator would fail or fragment it), or a latency-critical loop that cannot afford the
+// device-wide synchronisation an allocation implies.  mop_create allocates, so those callers
+// cannot hold a context.  For them the unit histogram of the permutation lives in the
+// file-scope device array below, which every GPU that loads this library holds until exit.
+// ---------------------------------------------------------------------------------------------
+#define MOP_STATIC_SCRATCH_INTS 262144   /* 1 MiB: ceil(T*k/512) * E entries must fit */
+static __device__ __align__(256) int32_t g_static_scratch[MOP_STATIC_SCRATCH_INTS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+struct StaticSetup { bool done; int32_t* scratch; int sm_count; };
+StaticSetup g_static_setup[kMaxDevices];   // zero-initialised
+std::mutex g_static_mutex;
+
+// Device address of g_static_scratch on `device` (which must be current).  In host code the
+// array's name is only a handle; the kernels need the address that cudaGetSymbolAddress returns
+// for the current device.
+mop_status static_setup(int device, StaticSetup* out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup& s = g_static_setup[device];
+    if (!s.done) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return MOP_ERR_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return MOP_ERR_CUDA;
+        s.scratch = static_cast<int32_t*>(ptr);
+        s.sm_count = sms;
+        s.done = true;
+    }
+    *out = s;
+    return MOP_OK;
+}
+}  // namespace
+
+mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, int32_t k, const void* x,
+                                  const int32_t* topk_idx, int32_t* counts, int32_t* offsets, int32_t* perm_row,
+                                  int32_t* row_src, void* Xp, void* stream) {
+    if (T < 0 || d < 1 || E < 1 || k < 1 || k > E) return MOP_ERR_INVALID_ARG;
+    if (d % 8) return MOP_ERR_ALIGN;
+    if (E > SEL_MAX_E || k > 32 || (long long)T * k >= (1ll << 31) - 4096) return MOP_ERR_SHAPE;
+    const int M = T * k;
+    const int units = ceil_div(M, PERM_SEG);
+    if ((long long)units * E > MOP_STATIC_SCRATCH_INTS) return MOP_ERR_SHAPE;   // beyond the static scratch
+    if (!counts || !offsets) return MOP_ERR_INVALID_ARG;
+    if (!aligned16(counts) || !aligned16(offsets)) return MOP_ERR_ALIGN;
+    if (T > 0) {
+        if (!x || !topk_idx || !perm_row || !row_src || !Xp) return MOP_ERR_INVALID_ARG;
+        if (!aligned16(x) || !aligned16(topk_idx) || !aligned16(perm_row) || !aligned16(row_src) || !aligned16(Xp))
+            return MOP_ERR_ALIGN;
+    }
+    if (device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    StaticSetup su;
+    mop_status r = static_setup(device, &su);
+    if (r != MOP_OK) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t smem = (size_t)PERM_WARPS * E * sizeof(int32_t);
+    // Nothing in the scratch has to start at zero: the histogram kernel writes every entry
+    // [unit][expert] that the scan and rank kernels read, so a previous call's contents are dead.
+    if (units > 0) perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, M, E);
+    perm_scan_kernel<<<1, 1024, (E + 1) * sizeof(int32_t), st>>>(su.scratch, counts, offsets, units, E);
+    if (units > 0) {
+        perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, perm_row,
+                                                                                    row_src, M, E);
+        const int blocks = min(ceil_div(T, 8), su.sm_count * 8);
+        scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, T,
+                                                    k, d / 8);
+    }
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
 }  // extern "C"
