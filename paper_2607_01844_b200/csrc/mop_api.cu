@@ -292,9 +292,7 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
     if (!guard.ok) return MOP_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* z = logits_opt ? logits_opt : c->z;
-    dim3 grid(ceil_div(s.T, SC_TT), ceil_div(s.E, SC_TE));
-    LAUNCH(c, "route_score", st,
-           route_score_kernel<<<grid, 256, 0, st>>>(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E));
+    LAUNCH(c, "route_score", st, route_score(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E, c->sm_count, st));
     mop_status r = after_launch(c);
     if (r != MOP_OK) return r;
     const size_t smem = (size_t)SEL_WARPS * 2 * s.E * sizeof(float);

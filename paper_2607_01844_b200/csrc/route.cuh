@@ -9,80 +9,176 @@ namespace mop {
 // Scoring.  z[t,e] = sum_i x[t,i] * W_r[i,e] as ONE chain of fused multiply-adds per (t,e), i
 // ascending, each step rounded once to fp32.  The chain order is part of the routing contract
 // (it makes top-k indices reproducible bit for bit), so there is no split over i and no tensor
-// core here; parallelism comes from the T*E independent chains.  Tile: 64 tokens x 64 experts
-// per 256-thread block, 4x4 chains per thread, operands staged through shared memory in slabs
-// of 32 along i.
+// core here; parallelism comes from the T*E independent chains and the kernel is bound by the
+// fp32 pipes.  Each thread owns RT tokens x RE experts (RT*RE chains) and advances two chains
+// per instruction with the packed fma.rn.f32x2 of sm_100 (two independent IEEE fused
+// multiply-adds: the rounding of each chain is unchanged).  A 128-thread CTA covers
+// (16 RT) tokens x (8 RE) experts; operands are staged through shared memory in slabs of 16 or 32
+// along i, double-buffered, the next slab prefetched into registers while the current one is
+// multiplied.  <8,8> needs 4 shared loads per 64 FMAs; smaller tiles trade that for more CTAs
+// when T*E is small.
 // ---------------------------------------------------------------------------------------------
-constexpr int SC_TT = 64, SC_TE = 64, SC_TK = 32;
+constexpr int SC_THREADS = 128;
 
-__global__ void __launch_bounds__(256) route_score_kernel(const bf16* __restrict__ x, const float* __restrict__ W_r,
-                                                          float* __restrict__ z, int T, int d, int E) {
-    __shared__ __align__(16) float xs[SC_TK][SC_TT + 4];
-    __shared__ __align__(16) float ws[SC_TK][SC_TE + 4];
-    const int t0 = blockIdx.x * SC_TT, e0 = blockIdx.y * SC_TE;
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+
+template <int RT, int RE, int SC_TK>
+__global__ void __launch_bounds__(SC_THREADS) route_score_kernel(const bf16* __restrict__ x,
+                                                                 const float* __restrict__ W_r,
+                                                                 float* __restrict__ z, int T, int d, int E) {
+    constexpr int TT = 16 * RT, TE = 8 * RE;          // CTA tile
+    constexpr int LDX = TT + 4, LDW = TE + 4;
+    constexpr int XV = TT * SC_TK / 8 / SC_THREADS;   // 16-byte x vectors fetched per thread per slab
+    constexpr int WV = TE * SC_TK / 4 / SC_THREADS;   // float4 W vectors per thread per slab
+    static_assert(RT % 2 == 0 && RE % 4 == 0 && XV >= 1 && WV >= 1, "tile shape");
+    __shared__ __align__(16) float xs[2][SC_TK][LDX];
+    __shared__ __align__(16) float ws[2][SC_TK][LDW];
+    const int t0 = blockIdx.x * TT, e0 = blockIdx.y * TE;
     const int tid = threadIdx.x;
-    const int tt = (tid / 16) * 4, te = (tid % 16) * 4;
-    float acc[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+    const int tt = (tid / 8) * RT, te = (tid % 8) * RE;
+    const bool w_vec = (E % 4 == 0);
 
-    for (int i0 = 0; i0 < d; i0 += SC_TK) {
-        // x slab: 64 tokens x 32 i  (each thread 8 elements: one token, 8 consecutive i)
-        {
-            const int tok = tid / 4, ii = (tid % 4) * 8;
-            const int t = t0 + tok;
-            float v[8];
+    unsigned long long acc[RT / 2][RE];   // acc[a][b] = chains of tokens (2a, 2a+1) for expert b
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = 0.0f;
-            if (t < T) {
-                if (i0 + ii + 8 <= d) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(x + (size_t)t * d + i0 + ii);
-                    v[0] = bf16_lo(raw.x); v[1] = bf16_hi(raw.x); v[2] = bf16_lo(raw.y); v[3] = bf16_hi(raw.y);
-                    v[4] = bf16_lo(raw.z); v[5] = bf16_hi(raw.z); v[6] = bf16_lo(raw.w); v[7] = bf16_hi(raw.w);
-                } else {
-                    for (int q = 0; q < 8; ++q)
-                        if (i0 + ii + q < d) v[q] = __bfloat162float(x[(size_t)t * d + i0 + ii + q]);
+    for (int a = 0; a < RT / 2; ++a)
+#pragma unroll
+        for (int b = 0; b < RE; ++b) acc[a][b] = 0ull;
+
+    uint4 xr[XV];
+    float4 wr[WV];
+    // x slab: TT tokens x SC_TK i, vector v of a thread = token lin / (SC_TK/8), i offset (lin % (SC_TK/8)) * 8
+    auto fetch = [&](int i0) {
+#pragma unroll
+        for (int v = 0; v < XV; ++v) {
+            const int lin = v * SC_THREADS + tid;
+            const int t = t0 + lin / (SC_TK / 8), i = i0 + (lin % (SC_TK / 8)) * 8;
+            xr[v] = (t < T && i < d) ? *reinterpret_cast<const uint4*>(x + (size_t)t * d + i) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int v = 0; v < WV; ++v) {
+            const int lin = v * SC_THREADS + tid;
+            const int i = i0 + lin / (TE / 4), e = e0 + (lin % (TE / 4)) * 4;
+            float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < d) {
+                const float* src = W_r + (size_t)i * E + e;
+                if (w_vec && e + 3 < E) q = *reinterpret_cast<const float4*>(src);
+                else {
+                    if (e < E) q.x = src[0];
+                    if (e + 1 < E) q.y = src[1];
+                    if (e + 2 < E) q.z = src[2];
+                    if (e + 3 < E) q.w = src[3];
                 }
             }
-#pragma unroll
-            for (int q = 0; q < 8; ++q) xs[ii + q][tok] = v[q];
+            wr[v] = q;
         }
-        // W_r slab: 32 i x 64 experts
+    };
+    auto stash = [&](int buf) {
 #pragma unroll
-        for (int r = 0; r < (SC_TK * SC_TE) / 256; ++r) {
-            const int lin = r * 256 + tid;
-            const int ii = lin / SC_TE, ee = lin % SC_TE;
-            float w = 0.0f;
-            if (i0 + ii < d && e0 + ee < E) w = W_r[(size_t)(i0 + ii) * E + e0 + ee];
-            ws[ii][ee] = w;
+        for (int v = 0; v < XV; ++v) {
+            const int lin = v * SC_THREADS + tid;
+            const int tok = lin / (SC_TK / 8), ii = (lin % (SC_TK / 8)) * 8;
+            const uint32_t w4[4] = {xr[v].x, xr[v].y, xr[v].z, xr[v].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                xs[buf][ii + 2 * q][tok] = bf16_lo(w4[q]);
+                xs[buf][ii + 2 * q + 1][tok] = bf16_hi(w4[q]);
+            }
         }
-        __syncthreads();
-        // Past-the-end i (d not a multiple of 32) contributes fma(0, 0, acc) = acc: exact.
-#pragma unroll 8
+#pragma unroll
+        for (int v = 0; v < WV; ++v) {
+            const int lin = v * SC_THREADS + tid;
+            *reinterpret_cast<float4*>(&ws[buf][lin / (TE / 4)][(lin % (TE / 4)) * 4]) = wr[v];
+        }
+    };
+
+    fetch(0);
+    stash(0);
+    __syncthreads();
+    int buf = 0;
+    for (int i0 = 0; i0 < d; i0 += SC_TK) {
+        const bool more = i0 + SC_TK < d;
+        if (more) fetch(i0 + SC_TK);
+        // Past-the-end i (d not a multiple of the slab) multiplies zeros: fma(0, 0, acc) = acc, exact.
+#pragma unroll
         for (int kk = 0; kk < SC_TK; ++kk) {
-            const float4 xv = *reinterpret_cast<const float4*>(&xs[kk][tt]);
-            const float4 wv = *reinterpret_cast<const float4*>(&ws[kk][te]);
-            const float xa[4] = {xv.x, xv.y, xv.z, xv.w};
-            const float wa[4] = {wv.x, wv.y, wv.z, wv.w};
+            unsigned long long xp[RT / 2], wp[RE];
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
+            for (int a = 0; a < RT / 4; ++a) {
+                const float4 v = *reinterpret_cast<const float4*>(&xs[buf][kk][tt + 4 * a]);
+                xp[2 * a] = pack_f32x2(v.x, v.y);
+                xp[2 * a + 1] = pack_f32x2(v.z, v.w);
+            }
+            if constexpr (RT % 4 == 2) {
+                const float2 v = *reinterpret_cast<const float2*>(&xs[buf][kk][tt + RT - 2]);
+                xp[RT / 2 - 1] = pack_f32x2(v.x, v.y);
+            }
 #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[a][b] = __fmaf_rn(xa[a], wa[b], acc[a][b]);
+            for (int b = 0; b < RE / 4; ++b) {
+                const float4 v = *reinterpret_cast<const float4*>(&ws[buf][kk][te + 4 * b]);
+                wp[4 * b] = pack_f32x2(v.x, v.x);
+                wp[4 * b + 1] = pack_f32x2(v.y, v.y);
+                wp[4 * b + 2] = pack_f32x2(v.z, v.z);
+                wp[4 * b + 3] = pack_f32x2(v.w, v.w);
+            }
+#pragma unroll
+            for (int a = 0; a < RT / 2; ++a)
+#pragma unroll
+                for (int b = 0; b < RE; ++b) fma_f32x2(acc[a][b], xp[a], wp[b]);
         }
+        if (more) stash(buf ^ 1);
         __syncthreads();
+        buf ^= 1;
     }
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
-        const int t = t0 + tt + a;
-        if (t >= T) continue;
+    for (int a = 0; a < RT / 2; ++a) {
+        float lo[RE], hi[RE];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int e = e0 + te + b;
-            if (e < E) z[(size_t)t * E + e] = acc[a][b];
+        for (int b = 0; b < RE; ++b) unpack_f32x2(acc[a][b], lo[b], hi[b]);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int t = t0 + tt + 2 * a + h;
+            if (t >= T) continue;
+            float* dst = z + (size_t)t * E + e0 + te;
+#pragma unroll
+            for (int b = 0; b < RE; b += 4) {
+                const float v0 = h ? hi[b] : lo[b], v1 = h ? hi[b + 1] : lo[b + 1];
+                const float v2 = h ? hi[b + 2] : lo[b + 2], v3 = h ? hi[b + 3] : lo[b + 3];
+                if (w_vec && e0 + te + b + 3 < E) {
+                    *reinterpret_cast<float4*>(dst + b) = make_float4(v0, v1, v2, v3);
+                } else {
+                    if (e0 + te + b < E) dst[b] = v0;
+                    if (e0 + te + b + 1 < E) dst[b + 1] = v1;
+                    if (e0 + te + b + 2 < E) dst[b + 2] = v2;
+                    if (e0 + te + b + 3 < E) dst[b + 3] = v3;
+                }
+            }
         }
     }
+}
+
+// Tile choice: the largest tile that still gives every SM a few CTAs.
+template <int RT, int RE, int TK>
+inline void launch_route_score(const bf16* x, const float* W_r, float* z, int T, int d, int E, cudaStream_t st) {
+    dim3 grid(ceil_div(T, 16 * RT), ceil_div(E, 8 * RE));
+    route_score_kernel<RT, RE, TK><<<grid, SC_THREADS, 0, st>>>(x, W_r, z, T, d, E);
+}
+inline void route_score(const bf16* x, const float* W_r, float* z, int T, int d, int E, int sm_count,
+                        cudaStream_t st) {
+    const long long big = (long long)ceil_div(T, 128) * ceil_div(E, 64);
+    const long long mid = (long long)ceil_div(T, 64) * ceil_div(E, 32);
+    if (big >= 2ll * sm_count) launch_route_score<8, 8, 16>(x, W_r, z, T, d, E, st);
+    else if (2 * mid >= sm_count) launch_route_score<4, 4, 32>(x, W_r, z, T, d, E, st);
+    else launch_route_score<2, 4, 32>(x, W_r, z, T, d, E, st);
 }
 
 // Sigmoid of the routing contract: a fixed sequence of fp32 operations, each rounded once
