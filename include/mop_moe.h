@@ -51,7 +51,13 @@ typedef enum { MOP_SCORE_SOFTMAX = 0, MOP_SCORE_SIGMOID = 1 } mop_score_fn;
  * gate numerator in POST_SCORE mode. */
 typedef enum { MOP_BIAS_NONE = 0, MOP_BIAS_POST_SCORE = 1, MOP_BIAS_PRE_LOGIT = 2 } mop_bias_mode;
 
-typedef enum { MOP_GEMM_AUTO = 0, MOP_GEMM_TENSOR = 1, MOP_GEMM_SCALAR = 2 } mop_gemm_path;
+/* AUTO: tensor cores when the shape allows, else scalar.  TENSOR: tensor cores or fail.  Both run
+ * the token-row GEMMs on the one-CTA kernel (128 x 256 tiles), the fastest schedule measured on
+ * every workload.  TENSOR_2CTA runs them on the two-CTA kernel (256 x 256 pair tiles; the last
+ * pair of an expert may be partly empty); TENSOR_MIXED sends the full 256-row pairs of every expert
+ * to the two-CTA kernel and the remaining rows to the one-CTA kernel. */
+typedef enum { MOP_GEMM_AUTO = 0, MOP_GEMM_TENSOR = 1, MOP_GEMM_SCALAR = 2, MOP_GEMM_TENSOR_1CTA = 3,
+               MOP_GEMM_TENSOR_2CTA = 4, MOP_GEMM_TENSOR_MIXED = 5 } mop_gemm_path;
 
 typedef struct {
     int32_t T, d, E, k, f;

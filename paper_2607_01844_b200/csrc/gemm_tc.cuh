@@ -284,6 +284,63 @@ __global__ void __launch_bounds__(1024) tc_build_mtiles_kernel(const int32_t* __
     if (e == 1023) *n_mtiles = scan[1023];
 }
 
+// Epilogue of one 128 x 256 accumulator for the kinds whose rows are token rows: this thread owns
+// row `grow` (valid iff row_ok) and walks the 256 columns in runs of 32.
+template <int KIND>
+__device__ __forceinline__ void tc_epilogue_rows(const TcArgs& args, uint32_t taddr, bool row_ok, int grow, int n0,
+                                                 int nt) {
+    float acc[32];
+    if constexpr (KIND == TC_F1) {
+        float acc2[32];
+#pragma unroll 1
+        for (int c = 0; c < 128; c += 32) {
+            tmem_ld32(taddr + c, acc);
+            tmem_ld32(taddr + 128 + c, acc2);
+            if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                for (int s = 0; s < 32; s += 8) {
+                    float g8[8], u8[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { g8[q] = acc[s + q]; u8[q] = acc2[s + q]; }
+                    epi_swiglu<8>(args.ep, grow, n0 + c + s, g8, u8);
+                }
+            }
+        }
+    } else if constexpr (KIND == TC_F2 || KIND == TC_B2) {
+        const float gate = row_ok ? args.ep.gate[args.ep.row_src[grow]] : 0.0f;
+        float dot = 0.0f;
+#pragma unroll 1
+        for (int c = 0; c < TC_BN; c += 32) {
+            tmem_ld32(taddr + c, acc);
+            if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                for (int s = 0; s < 32; s += 8) {
+                    float a8[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
+                    if constexpr (KIND == TC_F2) epi_gate<8>(args.ep, grow, n0 + c + s, gate, a8);
+                    else dot += epi_dh<8>(args.ep, grow, n0 + c + s, gate, a8);
+                }
+            }
+        }
+        if (KIND == TC_B2 && row_ok) args.ep.part[(size_t)nt * args.ep.M_total + grow] = dot;
+    } else if constexpr (KIND == TC_B4) {
+#pragma unroll 1
+        for (int c = 0; c < TC_BN; c += 32) {
+            tmem_ld32(taddr + c, acc);
+            if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                for (int s = 0; s < 32; s += 8) {
+                    float a8[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
+                    store_bf16_run<8>(args.ep.out0 + (size_t)grow * args.ep.ldo + n0 + c + s, a8);
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------ kernel
 template <int KIND>
 __global__ void __launch_bounds__(TcTraits<KIND>::THREADS, 1)
@@ -465,55 +522,10 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             const bool row_ok = Tr::RAGGED_K ? (ti.m0 + r < args.Mfix) : (r < ti.rows);
             const int grow = ti.row0 + r;        // ragged M: global row
             float acc[32];
+            (void)acc;
 
-            if constexpr (KIND == TC_F1) {
-                float acc2[32];
-#pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
-                    tmem_ld32(taddr + c, acc);
-                    tmem_ld32(taddr + 128 + c, acc2);
-                    if (row_ok && n0 + c < args.N) {
-#pragma unroll
-                        for (int s = 0; s < 32; s += 8) {
-                            float g8[8], u8[8];
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) { g8[q] = acc[s + q]; u8[q] = acc2[s + q]; }
-                            epi_swiglu<8>(args.ep, grow, n0 + c + s, g8, u8);
-                        }
-                    }
-                }
-            } else if constexpr (KIND == TC_F2 || KIND == TC_B2) {
-                const float gate = row_ok ? args.ep.gate[args.ep.row_src[grow]] : 0.0f;
-                float dot = 0.0f;
-#pragma unroll 1
-                for (int c = 0; c < TC_BN; c += 32) {
-                    tmem_ld32(taddr + c, acc);
-                    if (row_ok && n0 + c < args.N) {
-#pragma unroll
-                        for (int s = 0; s < 32; s += 8) {
-                            float a8[8];
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
-                            if constexpr (KIND == TC_F2) epi_gate<8>(args.ep, grow, n0 + c + s, gate, a8);
-                            else dot += epi_dh<8>(args.ep, grow, n0 + c + s, gate, a8);
-                        }
-                    }
-                }
-                if (KIND == TC_B2 && row_ok) args.ep.part[(size_t)ti.nt * args.ep.M_total + grow] = dot;
-            } else if constexpr (KIND == TC_B4) {
-#pragma unroll 1
-                for (int c = 0; c < TC_BN; c += 32) {
-                    tmem_ld32(taddr + c, acc);
-                    if (row_ok && n0 + c < args.N) {
-#pragma unroll
-                        for (int s = 0; s < 32; s += 8) {
-                            float a8[8];
-#pragma unroll
-                            for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
-                            store_bf16_run<8>(args.ep.out0 + (size_t)grow * args.ep.ldo + n0 + c + s, a8);
-                        }
-                    }
-                }
+            if constexpr (!Tr::RAGGED_K) {
+                tc_epilogue_rows<KIND>(args, taddr, row_ok, grow, n0, ti.nt);
             } else {
                 // Weight-gradient tile: each warp transposes 32 rows x 32 fp32 columns through shared
                 // memory (128-byte rows, 16-byte chunks XOR-swizzled by row: conflict-free both ways)
@@ -584,6 +596,7 @@ struct TcPlan {
     int sm_count;
     mop_moe_shape s;
     void* encode;   // cuTensorMapEncodeTiled
+    int pairs;      // 1: token-row kinds run as two-CTA pairs (256 x 256 tiles)
     Profiler* prof;
 };
 
@@ -698,96 +711,6 @@ inline mop_status tc_build_tiles(const TcPlan* p, const int32_t* offsets, int32_
     tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(offsets, p->s.E, reinterpret_cast<int4*>(tiles + 64), tiles);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
-}
-
-inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
-                             int* launches) {
-    const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
-    mop_status r;
-    if ((r = tc_build_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
-    ++*launches;
-    CUtensorMap mXp, mWg, mWu, mH, mWd;
-    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, 128) || !tc_map_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 64) ||
-        !tc_map_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 64) || !tc_map_2d(p, &mH, a.H, M, s.f, 128) ||
-        !tc_map_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 64))
-        return MOP_ERR_CUDA;
-    {   // F1: [G|U] = Xp [W_gate | W_up], SwiGLU epilogue
-        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
-        g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_F1>(p, "gemm_up_swiglu", mXp, mXp, mWg, mWu, mXp, mXp, g, st)) != MOP_OK) return r;
-        ++*launches;
-    }
-    {   // F2: Yp = gate * (H W_down)
-        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
-        g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_F2>(p, "gemm_down_gate", mH, mH, mWd, mWd, mH, mH, g, st)) != MOP_OK) return r;
-        ++*launches;
-    }
-    return MOP_OK;
-}
-
-inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
-                             int* launches, int* ntile_part) {
-    const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
-    *ntile_part = ceil_div(s.f, 256);
-    if (M == 0) {
-        // no rows at all: gradients are zero unless accumulating
-        if (!a.accumulate) {
-            const size_t n = (size_t)s.E * s.d * s.f * 4;
-            if (cudaMemsetAsync(a.dW_gate, 0, n, st) != cudaSuccess || cudaMemsetAsync(a.dW_up, 0, n, st) != cudaSuccess ||
-                cudaMemsetAsync(a.dW_down, 0, n, st) != cudaSuccess)
-                return MOP_ERR_CUDA;
-        }
-        return MOP_OK;
-    }
-    mop_status r;
-    if ((r = tc_build_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
-    ++*launches;
-    CUtensorMap mdYpA, mWdK, mdG, mdU, mWgK, mWuK, mgH, mdYpB, mXpA, mdGB, mdUB, moWd, moWg, moWu;
-    if (!tc_map_out_f32(p, &moWd, a.dW_down, s.E, s.f, s.d) || !tc_map_out_f32(p, &moWg, a.dW_gate, s.E, s.d, s.f) ||
-        !tc_map_out_f32(p, &moWu, a.dW_up, s.E, s.d, s.f))
-        return MOP_ERR_CUDA;
-    if (!tc_map_2d(p, &mdYpA, a.dYp, M, s.d, 128) || !tc_map_3d(p, &mWdK, a.W_down, s.E, s.f, s.d, 256) ||
-        !tc_map_2d(p, &mdG, a.dG, M, s.f, 128) || !tc_map_2d(p, &mdU, a.dU, M, s.f, 128) ||
-        !tc_map_3d(p, &mWgK, a.W_gate, s.E, s.d, s.f, 256) || !tc_map_3d(p, &mWuK, a.W_up, s.E, s.d, s.f, 256) ||
-        !tc_map_2d(p, &mgH, a.gH, M, s.f, 64) || !tc_map_2d(p, &mdYpB, a.dYp, M, s.d, 64) ||
-        !tc_map_2d(p, &mXpA, a.Xp, M, s.d, 64) || !tc_map_2d(p, &mdGB, a.dG, M, s.f, 64) ||
-        !tc_map_2d(p, &mdUB, a.dU, M, s.f, 64))
-        return MOP_ERR_CUDA;
-    {   // B2: dHu = dYp W_down^T, SwiGLU backward epilogue
-        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
-        g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
-        g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.part = a.part; g.ep.ldo = s.f; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_B2>(p, "gemm_dgrad_down_dswiglu", mdYpA, mdYpA, mWdK, mWdK, mdYpA, mdYpA, g, st)) != MOP_OK) return r;
-        ++*launches;
-    }
-    {   // B4: dXp = dG W_gate^T + dU W_up^T
-        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
-        g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_launch<TC_B4>(p, "gemm_dgrad_gate_up", mdG, mdU, mWgK, mWuK, mdG, mdG, g, st)) != MOP_OK) return r;
-        ++*launches;
-    }
-    {   // WD: dW_down[e] = (gate H)_e^T dYp_e
-        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.d, 256); g.tiles_m_fixed = ceil_div(s.f, TC_BM); g.Mfix = s.f; g.N = s.d;
-        g.ep.outf = a.dW_down; g.ep.accumulate = a.accumulate;
-        if ((r = tc_launch<TC_WD>(p, "gemm_wgrad_down", mgH, mgH, mdYpB, mdYpB, moWd, moWd, g, st)) != MOP_OK) return r;
-        ++*launches;
-    }
-    {   // WGU: [dW_gate | dW_up][e] = Xp_e^T [dG | dU]_e
-        TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.f, 128); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
-        g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate;
-        if ((r = tc_launch<TC_WGU>(p, "gemm_wgrad_gate_up", mXpA, mXpA, mdGB, mdUB, moWg, moWu, g, st)) != MOP_OK) return r;
-        ++*launches;
-    }
-    return MOP_OK;
 }
 
 }  // namespace mop

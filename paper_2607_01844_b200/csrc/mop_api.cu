@@ -11,7 +11,7 @@
 #include "common.cuh"
 #include "epilogue.cuh"
 #include "gemm_scalar.cuh"
-#include "gemm_tc.cuh"
+#include "gemm_host.cuh"
 #include "permute.cuh"
 #include "route.cuh"
 
@@ -61,7 +61,7 @@ Layout make_layout(const mop_moe_shape& s) {
     const size_t T = s.T, d = s.d, E = s.E, k = s.k, f = s.f, M = T * k;
     L.z = take(T * E * 4);
     L.partial = take((size_t)perm_units(s) * E * 4 + 4);
-    L.tiles = take(tc_tile_table_bytes(s.T * s.k, s.E));
+    L.tiles = take(tc_tables_bytes(s.T * s.k, s.E));
     L.status = take(256);
     if (s.with_backward) {
         L.part = take((size_t)part_tiles(s) * M * 4);
@@ -102,7 +102,7 @@ mop_status check_shape(const mop_moe_shape* s) {
     if (s->score_fn != MOP_SCORE_SOFTMAX && s->score_fn != MOP_SCORE_SIGMOID) return MOP_ERR_INVALID_ARG;
     if (s->bias_mode < MOP_BIAS_NONE || s->bias_mode > MOP_BIAS_PRE_LOGIT) return MOP_ERR_INVALID_ARG;
     if (s->bias_mode == MOP_BIAS_POST_SCORE && s->score_fn != MOP_SCORE_SIGMOID) return MOP_ERR_INVALID_ARG;
-    if (s->gemm_path < MOP_GEMM_AUTO || s->gemm_path > MOP_GEMM_SCALAR) return MOP_ERR_INVALID_ARG;
+    if (s->gemm_path < MOP_GEMM_AUTO || s->gemm_path > MOP_GEMM_TENSOR_MIXED) return MOP_ERR_INVALID_ARG;
     if ((long long)s->T * s->k >= (1ll << 31) - 4096) return MOP_ERR_SHAPE;
     if (s->E > SEL_MAX_E || s->k > 32) return MOP_ERR_SHAPE;
     if ((long long)s->T * s->d >= (1ll << 40) || (long long)s->d * s->f >= (1ll << 31)) return MOP_ERR_SHAPE;
@@ -205,7 +205,10 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return MOP_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
     c->tensor_ok = (prop.major == 10) && tc_shape_supported(shape->d, shape->f);
-    if (shape->gemm_path == MOP_GEMM_TENSOR && !c->tensor_ok) { delete c; return MOP_ERR_UNSUPPORTED; }
+    if ((shape->gemm_path == MOP_GEMM_TENSOR || shape->gemm_path >= MOP_GEMM_TENSOR_1CTA) && !c->tensor_ok) {
+        delete c;
+        return MOP_ERR_UNSUPPORTED;
+    }
     const Layout L = make_layout(*shape);
     c->ws_bytes = L.total;
     if (cudaMalloc(&c->ws, L.total) != cudaSuccess) { cudaGetLastError(); delete c; return MOP_ERR_WORKSPACE; }
@@ -245,7 +248,10 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
     if (cudaMemset(c->status, 0, 256) != cudaSuccess) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
     if (c->tensor_ok) {
         st = tc_plan_init(&c->plan, *shape, c->sm_count, &c->prof);
+        if (st == MOP_OK) st = tc2_init();
         if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
+        c->plan.pairs = shape->gemm_path == MOP_GEMM_TENSOR_2CTA ? 1 : shape->gemm_path == MOP_GEMM_TENSOR_MIXED ? 2 : 0;
+        if (c->sm_count < 2) c->plan.pairs = 0;
     }
     *out = c;
     return MOP_OK;

@@ -110,6 +110,15 @@ def test_small_layers_match_oracle(w, path):
     check_layer(w, path)
 
 
+@pytest.mark.parametrize("path", [binding.GEMM_TENSOR_2CTA, binding.GEMM_TENSOR_MIXED], ids=["2cta", "mixed"])
+def test_two_cta_schedules_match_oracle_and_the_one_cta_kernel(path):
+    w = synth.small("c2_mid", T=1500, d=256, E=6, k=2, f=320, backward=True, seed=21)   # 500 rows per expert
+    _, buf = check_layer(w, path)
+    _, _, _, ref = run(w, binding.GEMM_TENSOR_1CTA)
+    for n in ("H", "Yp", "Y", "dX", "dgate", "dW_gate", "dW_up", "dW_down"):   # same accumulation order
+        assert torch.equal(getattr(buf, n), getattr(ref, n)), n
+
+
 def test_all_keys_equal_goes_to_lowest_ids_and_leaves_experts_empty():
     w = synth.small("c1_tiny", T=96, d=64, E=6, k=2, f=64, backward=True, seed=17)
     host = synth.make_inputs(w, "cpu")
