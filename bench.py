@@ -207,6 +207,7 @@ def main():
     ap.add_argument("--shape", default=None,
                     help="T,d,E,k,f overriding the named workload's sizes (same distributions): small cases for "
                          "profiler captures")
+    ap.add_argument("--gemm-path", type=int, default=0, help="mop_gemm_path (0 = library default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -239,7 +240,7 @@ def main():
             dist.barrier()
 
     inp = synth.make_inputs(w, dev)
-    ctx = binding.context_for(w, device=local, host_io=not args.no_e2e)
+    ctx = binding.context_for(w, device=local, host_io=not args.no_e2e, gemm_path=args.gemm_path)
     buf = binding.LayerBuffers(w, device=dev)
     stream = torch.cuda.current_stream()
 

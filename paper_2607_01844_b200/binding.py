@@ -17,7 +17,7 @@ LIB_PATH = _PKG / "libmop_moe.so"
 MOP_OK = 0
 STATUS_NAMES = {0: "MOP_OK", 1: "MOP_ERR_INVALID_ARG", 2: "MOP_ERR_SHAPE", 3: "MOP_ERR_ALIGN", 4: "MOP_ERR_WORKSPACE",
                 5: "MOP_ERR_CUDA", 6: "MOP_ERR_UNSUPPORTED", 7: "MOP_ERR_TIMEOUT"}
-GEMM_AUTO, GEMM_TENSOR, GEMM_SCALAR, GEMM_TENSOR_1CTA, GEMM_TENSOR_2CTA, GEMM_TENSOR_MIXED = 0, 1, 2, 3, 4, 5
+GEMM_AUTO, GEMM_TENSOR, GEMM_SCALAR, GEMM_TENSOR_1CTA, GEMM_TENSOR_2CTA, GEMM_TENSOR_MIXED, GEMM_TENSOR_TN = 0, 1, 2, 3, 4, 5, 6
 
 
 class MopShape(ctypes.Structure):

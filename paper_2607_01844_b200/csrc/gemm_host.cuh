@@ -2,13 +2,14 @@
 #pragma once
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
+#include "gemm_tn.cuh"
 
 namespace mop {
 
 // Schedules of the token-row kinds (TcPlan::pairs): 0 = one-CTA kernel on 128-row tiles; 1 = two-CTA
 // kernel on 256-row pairs (the last pair of an expert may be partly empty); 2 = mixed: full pairs on
 // the two-CTA kernel, the remaining < 256 rows of each expert on the one-CTA kernel.
-inline size_t tc_tables_bytes(int M, int E) { return 2 * tc_tile_table_bytes(M, E); }
+inline size_t tc_tables_bytes(int M, int E) { return 3 * tc_tile_table_bytes(M, E); }
 
 inline mop_status tc_build_row_tiles(const TcPlan* p, const int32_t* offsets, int32_t* tiles, cudaStream_t st) {
     int32_t* tiles2 = tiles + tc_tile_table_bytes(p->s.T * p->s.k, p->s.E) / 4;
@@ -46,25 +47,42 @@ inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int3
     const mop_moe_shape& s = p->s;
     const uint64_t M = (uint64_t)s.T * s.k;
     mop_status r;
-    if ((r = tc_build_row_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
-    ++*launches;
-    CUtensorMap mXp, mWg, mWu, mH, mWd;
-    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, 128) || !tc_map_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 64) ||
-        !tc_map_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 64) || !tc_map_2d(p, &mH, a.H, M, s.f, 128) ||
-        !tc_map_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 64))
+    // Tokens-on-N kernels: fwd_tn bit 0 = up-projection, bit 1 = down-projection (see tc_plan_policy)
+    const bool tn_f1 = p->fwd_tn & 1, tn_f2 = p->fwd_tn & 2;
+    if (tn_f1 || tn_f2) {
+        if ((r = tn_build_tiles(p, a.offsets, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    if (!tn_f1 || !tn_f2) {
+        if ((r = tc_build_row_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    // N-major weights as chunked maps: one-CTA tiles take 2 chunks per tensor (gate | up) or 4 (down);
+    // a pair CTA takes 2 chunks
+    CUtensorMap mXp, mWg, mWu, mH, mWd, mWdp;
+    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, 128) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 2) ||
+        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 2) || !tc_map_2d(p, &mH, a.H, M, s.f, 128) ||
+        !tc_map_chunked_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 4) ||
+        !tc_map_chunked_3d(p, &mWdp, a.W_down, s.E, s.f, s.d, 2))
         return MOP_ERR_CUDA;
-    {   // F1: [G|U] = Xp [W_gate | W_up], SwiGLU epilogue
+    if (tn_f1) {
+        if ((r = tn_up_swiglu(p, a, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), status, st)) != MOP_OK) return r;
+        ++*launches;
+    } else {   // F1: [G|U] = Xp [W_gate | W_up], SwiGLU epilogue
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
         g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
         if ((r = tc_rows_gemm<TC_F1>(p, "gemm_up_swiglu", "gemm_up_swiglu_2cta", mXp, mXp, mWg, mWu, mWg, mWu, g, tiles, st, launches)) != MOP_OK)
             return r;
     }
-    {   // F2: Yp = gate * (H W_down)
+    if (tn_f2) {
+        if ((r = tn_down_gate(p, a, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), status, st)) != MOP_OK) return r;
+        ++*launches;
+    } else {   // F2: Yp = gate * (H W_down)
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
         g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
-        if ((r = tc_rows_gemm<TC_F2>(p, "gemm_down_gate", "gemm_down_gate_2cta", mH, mH, mWd, mWd, mWd, mWd, g, tiles, st, launches)) != MOP_OK)
+        if ((r = tc_rows_gemm<TC_F2>(p, "gemm_down_gate", "gemm_down_gate_2cta", mH, mH, mWd, mWd, mWdp, mWdp, g, tiles, st, launches)) != MOP_OK)
             return r;
     }
     return MOP_OK;
@@ -99,9 +117,9 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
     if (!tc_map_2d(p, &mdYpA, a.dYp, M, s.d, 128) || !tc_map_3d(p, &mWdK, a.W_down, s.E, s.f, s.d, 256) ||
         !tc_map_2d(p, &mdG, a.dG, M, s.f, 128) || !tc_map_2d(p, &mdU, a.dU, M, s.f, 128) ||
         !tc_map_3d(p, &mWgK, a.W_gate, s.E, s.d, s.f, 256) || !tc_map_3d(p, &mWuK, a.W_up, s.E, s.d, s.f, 256) ||
-        !tc_map_2d(p, &mgH, a.gH, M, s.f, 64) || !tc_map_2d(p, &mdYpB, a.dYp, M, s.d, 64) ||
-        !tc_map_2d(p, &mXpA, a.Xp, M, s.d, 64) || !tc_map_2d(p, &mdGB, a.dG, M, s.f, 64) ||
-        !tc_map_2d(p, &mdUB, a.dU, M, s.f, 64))
+        !tc_map_chunked_2d(p, &mgH, a.gH, M, s.f, 2) || !tc_map_chunked_2d(p, &mdYpB, a.dYp, M, s.d, 4) ||
+        !tc_map_chunked_2d(p, &mXpA, a.Xp, M, s.d, 2) || !tc_map_chunked_2d(p, &mdGB, a.dG, M, s.f, 2) ||
+        !tc_map_chunked_2d(p, &mdUB, a.dU, M, s.f, 2))
         return MOP_ERR_CUDA;
     {   // B2: dHu = dYp W_down^T, SwiGLU backward epilogue
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);

@@ -146,6 +146,13 @@ __device__ __forceinline__ void tma_store_wait_read() {
 }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
+                                            int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, "
+        "%6}], [%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -410,19 +417,21 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                     if constexpr (!Tr::A_MN) {
                         tma_load_2d(sA, ph ? &tmA1 : &tmA0, fb, k0, ti.row0);
                     } else {
-                        const int krow = ti.row0 + kb * TC_BK;
-                        tma_load_2d(sA, &tmA0, fb, ti.m0, krow);
-                        tma_load_2d(sA + TC_CHUNK_BYTES, &tmA0, fb, ti.m0 + 64, krow);
+                        // chunked map {64, rows, cols/64}: both 64-wide column chunks in one copy
+                        tma_load_3d(sA, &tmA0, fb, 0, ti.row0 + kb * TC_BK, ti.m0 >> 6);
                     }
                     if constexpr (!Tr::B_MN) {
                         tma_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0, n0, ti.e);
                     } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const CUtensorMap* mp = (Tr::DUAL_B && c >= 2) ? &tmB1 : &tmB0;
-                            const int n = Tr::DUAL_B ? n0 + 64 * (c & 1) : n0 + 64 * c;
-                            if constexpr (Tr::B_WEIGHT) tma_load_3d(sB + c * TC_CHUNK_BYTES, mp, fb, n, k0, ti.e);
-                            else tma_load_2d(sB + c * TC_CHUNK_BYTES, mp, fb, n, ti.row0 + kb * TC_BK);
+                        // chunked maps {64, rows, cols/64 [, E]}: the 64-wide column chunks of the tile arrive
+                        // chunk-major in one copy per tensor (four chunks, or two each of two tensors)
+                        if constexpr (Tr::B_WEIGHT) {
+                            tma_load_4d(sB, &tmB0, fb, 0, k0, n0 >> 6, ti.e);
+                            if constexpr (Tr::DUAL_B) tma_load_4d(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, k0, n0 >> 6, ti.e);
+                        } else {
+                            const int krow = ti.row0 + kb * TC_BK;
+                            tma_load_3d(sB, &tmB0, fb, 0, krow, n0 >> 6);
+                            if constexpr (Tr::DUAL_B) tma_load_3d(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, krow, n0 >> 6);
                         }
                     }
                     if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
@@ -596,7 +605,8 @@ struct TcPlan {
     int sm_count;
     mop_moe_shape s;
     void* encode;   // cuTensorMapEncodeTiled
-    int pairs;      // 1: token-row kinds run as two-CTA pairs (256 x 256 tiles)
+    int pairs;      // schedule of the token-row kinds (see gemm_host.cuh)
+    int fwd_tn;     // forward GEMMs on the tokens-on-N kernels: bit 0 up-projection, bit 1 down-projection
     Profiler* prof;
 };
 
@@ -667,6 +677,33 @@ inline bool tc_map_3d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_
     const cuuint32_t box[3] = {64, box_rows, 1};
     const cuuint32_t es[3] = {1, 1, 1};
     return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Chunked maps for MN-major operands.  A dense [rows, cols] (or [E, rows, cols]) bf16 matrix is viewed
+// as {64 columns, rows, cols/64 chunks [, E]} so that ONE copy brings `chunks` 64-wide column chunks
+// of 64 rows each, chunk-major in shared memory: exactly the layout the MMA descriptor expects
+// (chunk pitch 8 KiB, 128-byte swizzled rows).  cols must be a multiple of 64.
+inline bool tc_map_chunked_2d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                              uint32_t chunks) {
+    const cuuint64_t dims[3] = {64, rows, cols / 64};
+    const cuuint64_t strides[2] = {cols * 2, 128};
+    const cuuint32_t box[3] = {64, 64, chunks};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+inline bool tc_map_chunked_3d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows,
+                              uint64_t cols, uint32_t chunks) {
+    const cuuint64_t dims[4] = {64, rows, cols / 64, E};
+    const cuuint64_t strides[3] = {cols * 2, 128, rows * cols * 2};
+    const cuuint32_t box[4] = {64, 64, chunks, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base),
                                                      dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;

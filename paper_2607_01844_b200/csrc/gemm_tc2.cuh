@@ -46,6 +46,13 @@ __device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* ma
         "%5}], [%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+__device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z,
+                                             int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, "
+        "%5, %6}], [%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
 __device__ __forceinline__ void tmem2_alloc(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
                  : "memory");
@@ -213,8 +220,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
                         // leader holds the gate columns and the peer the up columns
                         const CUtensorMap* mp = (Tr::DUAL_B && rank) ? &tmB1 : &tmB0;
                         const int nb = Tr::DUAL_B ? n0 : n0 + 128 * (int)rank;
-                        tma2_load_3d(sB, mp, fb, nb, k0, ti.e);
-                        tma2_load_3d(sB + TC_CHUNK_BYTES, mp, fb, nb + 64, k0, ti.e);
+                        tma2_load_4d(sB, mp, fb, 0, k0, nb >> 6, ti.e);   // chunked map, two chunks per copy
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }

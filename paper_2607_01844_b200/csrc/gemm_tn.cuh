@@ -1,0 +1,369 @@
+// "Tokens on N" two-CTA grouped GEMMs for the forward pass: the MMA computes the TRANSPOSED product
+//     D^T [weight rows (M = 256 across the CTA pair) x tokens (N <= 256)] = W^T-tile * Xp^T
+// so that the ragged dimension (an expert's token count) sits on the MMA's N, whose granularity is
+// 16, instead of on M, whose granularity is 128: an expert with 171 rows costs one N = 176 tile
+// instead of two 128-row tiles.  The weights are the "A" operand (each CTA of the pair holds its
+// own 128 weight rows), the tokens the "B" operand (each CTA loads half of the tile's token rows),
+// tcgen05.mma.cta_group::2 multiplies, and each CTA's TMEM receives [its 128 weight rows x N].
+//
+//   TN_F1  G^T|U^T: a CTA's 128 weight rows are 64 gate columns followed by the 64 matching up
+//          columns of W_gate / W_up, so G and U of one (f, token) land in the same CTA (TMEM lanes
+//          l and l + 64); the epilogue exchanges U through shared memory, applies SwiGLU and
+//          writes H (+ G, U stash) back in token-major layout.
+//   TN_F2  O^T = W_down^T-tile * H^T, gate applied per token column, Yp written token-major.
+//
+// The epilogue transposes 32 x 32 blocks through shared memory so that global stores are 64-byte
+// row segments.  Barrier protocol, bounded waits and teardown as in the pair kernel.
+#pragma once
+#include "gemm_tc2.cuh"
+
+namespace mop {
+
+enum : int { TN_F1 = 0, TN_F2 = 1 };
+
+constexpr int TN_STAGES = 5;
+constexpr int TN_A_BYTES = 128 * TC_BK * 2;          // 16 KiB: this CTA's 128 weight rows
+constexpr int TN_B_BYTES = 128 * TC_BK * 2;          // up to 128 token rows (half of N = 256)
+constexpr int TN_STAGE_BYTES = TN_A_BYTES + TN_B_BYTES;
+constexpr int TN_EPI_BYTES = 4 * 8192;               // per epilogue warp: transposition buffers
+constexpr int TN_SMEM_BYTES = TN_STAGES * TN_STAGE_BYTES + 1024 /*align*/ + TC_BAR_BYTES + TN_EPI_BYTES;
+constexpr int TN_THREADS = 192;
+constexpr int TN_BOX_ROWS = 128;                     // token rows per TMA box (one box per stage)
+
+struct TnArgs {
+    const int4* ttiles;       // {expert, first row, rows (1..256), 0} per token tile
+    const int32_t* n_ttiles;  // device scalar
+    int tiles_m;              // weight-row tiles per token tile (each 256 rows; F1: 128 columns of f)
+    int kblocks;              // K / 64 rounded up
+    int Mw;                   // weight rows in total (F1: f; F2: d)
+    int32_t* status;
+    EpiArgs ep;
+};
+
+// Token tiles: an expert's rows are cut into ceil(rows/256) nearly equal tiles.
+__global__ void __launch_bounds__(1024) tn_build_ttiles_kernel(const int32_t* __restrict__ offsets, int E,
+                                                               int4* __restrict__ tiles,
+                                                               int32_t* __restrict__ n_tiles) {
+    __shared__ int32_t scan[1024];
+    const int e = threadIdx.x;
+    int cnt = 0, off = 0;
+    if (e < E) { off = offsets[e]; cnt = offsets[e + 1] - off; }
+    const int nt = (cnt + 255) / 256;
+    scan[e] = nt;
+    __syncthreads();
+    for (int s = 1; s < 1024; s <<= 1) {
+        const int v = (e >= s) ? scan[e - s] : 0;
+        __syncthreads();
+        scan[e] += v;
+        __syncthreads();
+    }
+    const int first = scan[e] - nt;
+    const int sz = nt ? (((cnt + nt - 1) / nt + 15) & ~15) : 0;
+    for (int i = 0; i < nt; ++i) tiles[first + i] = make_int4(e, off + i * sz, min(sz, cnt - i * sz), 0);
+    if (e == 1023) *n_tiles = scan[1023];
+}
+
+__device__ __forceinline__ void bar_pair_sync(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
+
+// 32 tokens x 32 features staged as bf16 [token][feature] -> 64-byte row segments in global memory
+__device__ __forceinline__ void tn_write_rows(bf16* __restrict__ dst, int ldo, const uint16_t* st, int row0,
+                                              int rows_left, int col0, int lane) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int tok = 8 * i + (lane >> 2), part = lane & 3;
+        const uint4 v = *reinterpret_cast<const uint4*>(st + tok * 32 + part * 8);
+        if (tok < rows_left) *reinterpret_cast<uint4*>(dst + (size_t)(row0 + tok) * ldo + col0 + part * 8) = v;
+    }
+}
+
+__device__ __forceinline__ uint16_t bf16_bits(float v) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+
+template <int KIND>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TN_THREADS, 1)
+tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
+               const __grid_constant__ CUtensorMap tmB, const TnArgs args) {
+    constexpr int S = TN_STAGES;
+    extern __shared__ uint8_t tc_smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S * TN_STAGE_BYTES);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint8_t* epi_smem = smem + S * TN_STAGE_BYTES + TC_BAR_BYTES;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * S + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB);
+        if (KIND == TN_F1) tma_prefetch_desc(&tmA1);
+    }
+    if (warp == 1) tmem2_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int total_tiles = (*args.n_ttiles) * args.tiles_m;
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    // work tile t -> token tile t / tiles_m (its expert, first row, rows) and weight-row tile t % tiles_m
+    struct Tile { int e, row0, rows, nmma, mt; };
+    auto decode = [&](int t) {
+        const int4 m = __ldg(args.ttiles + t / args.tiles_m);
+        Tile ti;
+        ti.e = m.x; ti.row0 = m.y; ti.rows = m.z; ti.nmma = (m.z + 15) & ~15; ti.mt = t % args.tiles_m;
+        return ti;
+    };
+
+    if (warp == 0) {
+        // ===================================================================== TMA producer (both CTAs)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0; bool alive = true;
+            Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
+            for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
+                const Tile ti = nxt;
+                if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
+                const int half = ti.nmma >> 1;                         // token rows per CTA
+                const int nbox = (half + TN_BOX_ROWS - 1) / TN_BOX_ROWS;
+                const int brow0 = ti.row0 + (int)rank * half;
+                const uint32_t tx = 2u * (TN_A_BYTES + (uint32_t)nbox * TN_BOX_ROWS * 128u);
+                for (int kb = 0; kb < args.kblocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) {
+                        alive = false; break;
+                    }
+                    const uint32_t fb = full_bar(stage) & T2_PEER_MASK;
+                    if (leader) mbar_expect_tx(full_bar(stage), tx);
+                    const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
+                    const uint32_t sB = sA + TN_A_BYTES;
+                    const int k0 = kb * TC_BK;
+                    if constexpr (KIND == TN_F1) {
+                        // 64 gate columns, then the 64 matching up columns (N-major weights [E, d, f])
+                        const int f0 = ti.mt * 128 + 64 * (int)rank;
+                        tma2_load_4d(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e);
+                        tma2_load_4d(sA + TC_CHUNK_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e);
+                    } else {
+                        const int m0 = ti.mt * 256 + 128 * (int)rank;
+                        tma2_load_4d(sA, &tmA0, fb, 0, k0, m0 >> 6, ti.e);   // two chunks in one copy
+                    }
+                    for (int b = 0; b < nbox; ++b)
+                        tma2_load_2d(sB + b * TN_BOX_ROWS * 128, &tmB, fb, k0, brow0 + b * TN_BOX_ROWS);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================================================================== MMA issuer (leader CTA)
+        if (leader) {
+            int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
+            Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
+            for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
+                const Tile ti = nxt;
+                if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
+                // A is M-major (N-major weights), B is K-major; M = 256 over the pair, N = this tile's tokens
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) |
+                                       ((uint32_t)(ti.nmma >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+                const int buf = it & 1;
+                const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait_warp(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY, lane))
+                    break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * 256;
+                for (int kb = 0; kb < args.kblocks; ++kb) {
+                    if (!mbar_wait_warp(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL, lane)) {
+                        alive = false; break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
+                    const uint32_t sB = sA + TN_A_BYTES;
+                    if (lane == 0) {
+#pragma unroll
+                        for (int k4 = 0; k4 < TC_BK / 16; ++k4)
+                            umma2_bf16(d_tmem, smem_desc(sA + k4 * 2048, TC_CHUNK_BYTES, 1024),
+                                       smem_desc(sB + k4 * 32, 0, 1024), idesc, (kb | k4) != 0 ? 1u : 0u);
+                        umma2_commit_both(empty_bar(stage));
+                    }
+                    __syncwarp();
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                if (!alive) break;
+                if (lane == 0) umma2_commit_both(tfull_bar(buf));
+                __syncwarp();
+                ++it;
+            }
+        }
+    } else {
+        // ===================================================================== epilogue (4 warps, both CTAs)
+        const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+        uint8_t* wbuf = epi_smem + quarter * 8192;    // this warp's staging
+        int it = 0;
+        Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
+        for (int t = cluster_id; t < total_tiles; t += n_clusters) {
+            const Tile ti = nxt;
+            if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
+            const int buf = it & 1;
+            const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
+            if (!mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256;
+            float v[32];
+
+            if constexpr (KIND == TN_F1) {
+                // lanes 0..63 of the CTA hold gate rows, lanes 64..127 the matching up rows
+                const bool is_up = quarter >= 2;
+                const int fcol = ti.mt * 128 + 64 * (int)rank + 32 * (quarter & 1);   // first f of this warp
+                const bool f_ok = fcol < args.Mw;
+                float* ubuf = reinterpret_cast<float*>(epi_smem + (2 + (quarter & 1)) * 8192);   // in the up warp's region
+                // up warps: [32 x 33 fp32 exchange buffer | one bf16 block]; gate warps: two bf16 blocks
+                uint16_t* st0 = reinterpret_cast<uint16_t*>(is_up ? wbuf + 4352 : wbuf);
+                uint16_t* st1 = st0 + 1024;
+                const int pair_bar = 1 + (quarter & 1);
+#pragma unroll 1
+                for (int c = 0; c < ti.nmma; c += 32) {
+                    tmem_ld32(taddr + c, v);
+                    const int rows_left = ti.rows - c;
+                    if (is_up) {
+#pragma unroll
+                        for (int tk = 0; tk < 32; ++tk) ubuf[tk * 33 + lane] = v[tk];
+                        if (args.ep.out2) {
+#pragma unroll
+                            for (int tk = 0; tk < 32; ++tk) st0[tk * 32 + lane] = bf16_bits(v[tk]);
+                        }
+                        bar_pair_sync(pair_bar);     // U is in shared memory
+                        if (args.ep.out2 && f_ok) {
+                            __syncwarp();
+                            tn_write_rows(args.ep.out2, args.ep.ldo, st0, ti.row0 + c, rows_left, fcol, lane);
+                        }
+                        bar_pair_sync(pair_bar);     // the gate warp has read U
+                    } else {
+                        bar_pair_sync(pair_bar);
+#pragma unroll
+                        for (int tk = 0; tk < 32; ++tk) {
+                            const float u = ubuf[tk * 33 + lane];
+                            const float g = v[tk];
+                            st0[tk * 32 + lane] = bf16_bits(g * sigmoidf_acc(g) * u);
+                            if (args.ep.out1) st1[tk * 32 + lane] = bf16_bits(g);
+                        }
+                        __syncwarp();
+                        if (f_ok) {
+                            tn_write_rows(args.ep.out0, args.ep.ldo, st0, ti.row0 + c, rows_left, fcol, lane);
+                            if (args.ep.out1)
+                                tn_write_rows(args.ep.out1, args.ep.ldo, st1, ti.row0 + c, rows_left, fcol, lane);
+                        }
+                        bar_pair_sync(pair_bar);
+                    }
+                    __syncwarp();
+                }
+            } else {
+                const int mcol = ti.mt * 256 + 128 * (int)rank + 32 * quarter;      // first output column of this warp
+                const bool m_ok = mcol < args.Mw;
+                uint16_t* st0 = reinterpret_cast<uint16_t*>(wbuf);
+#pragma unroll 1
+                for (int c = 0; c < ti.nmma; c += 32) {
+                    tmem_ld32(taddr + c, v);
+                    const int rows_left = ti.rows - c;
+                    // gate of token (c + lane), handed round by shuffle
+                    float gmine = 0.0f;
+                    if (lane < rows_left) gmine = args.ep.gate[args.ep.row_src[ti.row0 + c + lane]];
+#pragma unroll
+                    for (int tk = 0; tk < 32; ++tk) {
+                        const float g = __shfl_sync(0xffffffffu, gmine, tk);
+                        st0[tk * 32 + lane] = bf16_bits(g * v[tk]);
+                    }
+                    __syncwarp();
+                    if (m_ok) tn_write_rows(args.ep.out0, args.ep.ldo, st0, ti.row0 + c, rows_left, mcol, lane);
+                    __syncwarp();
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tempty_bar(buf) & T2_PEER_MASK);
+            ++it;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) __nanosleep(1000);
+        __syncthreads();
+    }
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem2_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host
+inline mop_status tn_init() {
+    if (cudaFuncSetAttribute(tn_gemm_kernel<TN_F1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(tn_gemm_kernel<TN_F2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
+            cudaSuccess)
+        return MOP_ERR_CUDA;
+    return MOP_OK;
+}
+
+inline mop_status tn_build_tiles(TcPlan* p, const int32_t* offsets, int32_t* tiles, cudaStream_t st) {
+    p->prof->begin("tn_build_ttiles", st);
+    tn_build_ttiles_kernel<<<1, 1024, 0, st>>>(offsets, p->s.E, reinterpret_cast<int4*>(tiles + 64), tiles);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+inline TnArgs tn_base_args(int32_t* tiles, int32_t* status) {
+    TnArgs g{};
+    g.ttiles = reinterpret_cast<const int4*>(tiles + 64);
+    g.n_ttiles = tiles;
+    g.status = status;
+    return g;
+}
+
+// Up-projection + SwiGLU on the tokens-on-N kernel (`tiles` holds the token-tile table).
+inline mop_status tn_up_swiglu(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
+    const mop_moe_shape& s = p->s;
+    const uint64_t M = (uint64_t)s.T * s.k;
+    CUtensorMap mXp, mWg, mWu;
+    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1) ||
+        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1))
+        return MOP_ERR_CUDA;
+    TnArgs g = tn_base_args(tiles, status);
+    g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
+    g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
+    p->prof->begin("gemm_up_swiglu", st);
+    tn_gemm_kernel<TN_F1><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mXp, g);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+// Down-projection + gate on the tokens-on-N kernel.
+inline mop_status tn_down_gate(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
+    const mop_moe_shape& s = p->s;
+    const uint64_t M = (uint64_t)s.T * s.k;
+    CUtensorMap mH, mWd;
+    if (!tc_map_2d(p, &mH, a.H, M, s.f, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 2))
+        return MOP_ERR_CUDA;
+    TnArgs g = tn_base_args(tiles, status);
+    g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.Mw = s.d;
+    g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
+    p->prof->begin("gemm_down_gate", st);
+    tn_gemm_kernel<TN_F2><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWd, mWd, mH, g);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+}  // namespace mop

@@ -102,7 +102,7 @@ mop_status check_shape(const mop_moe_shape* s) {
     if (s->score_fn != MOP_SCORE_SOFTMAX && s->score_fn != MOP_SCORE_SIGMOID) return MOP_ERR_INVALID_ARG;
     if (s->bias_mode < MOP_BIAS_NONE || s->bias_mode > MOP_BIAS_PRE_LOGIT) return MOP_ERR_INVALID_ARG;
     if (s->bias_mode == MOP_BIAS_POST_SCORE && s->score_fn != MOP_SCORE_SIGMOID) return MOP_ERR_INVALID_ARG;
-    if (s->gemm_path < MOP_GEMM_AUTO || s->gemm_path > MOP_GEMM_TENSOR_MIXED) return MOP_ERR_INVALID_ARG;
+    if (s->gemm_path < MOP_GEMM_AUTO || s->gemm_path > MOP_GEMM_TENSOR_TN) return MOP_ERR_INVALID_ARG;
     if ((long long)s->T * s->k >= (1ll << 31) - 4096) return MOP_ERR_SHAPE;
     if (s->E > SEL_MAX_E || s->k > 32) return MOP_ERR_SHAPE;
     if ((long long)s->T * s->d >= (1ll << 40) || (long long)s->d * s->f >= (1ll << 31)) return MOP_ERR_SHAPE;
@@ -249,9 +249,18 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
     if (c->tensor_ok) {
         st = tc_plan_init(&c->plan, *shape, c->sm_count, &c->prof);
         if (st == MOP_OK) st = tc2_init();
+        if (st == MOP_OK) st = tn_init();
         if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
         c->plan.pairs = shape->gemm_path == MOP_GEMM_TENSOR_2CTA ? 1 : shape->gemm_path == MOP_GEMM_TENSOR_MIXED ? 2 : 0;
         if (c->sm_count < 2) c->plan.pairs = 0;
+        // Measured policy (B200): the tokens-on-N down-projection wins on every workload; the tokens-on-N
+        // up-projection wins when the K loop is long enough to hide its heavier epilogue (d >= 4096).
+        c->plan.fwd_tn = 0;
+        if (c->sm_count >= 2) {
+            if (shape->gemm_path == MOP_GEMM_TENSOR_TN) c->plan.fwd_tn = 3;
+            else if (shape->gemm_path == MOP_GEMM_AUTO || shape->gemm_path == MOP_GEMM_TENSOR)
+                c->plan.fwd_tn = 2 | (shape->d >= 4096 ? 1 : 0);
+        }
     }
     *out = c;
     return MOP_OK;

@@ -105,12 +105,19 @@ SMALL = [
 
 
 @pytest.mark.parametrize("w", SMALL, ids=lambda w: f"{w.name}-T{w.T}d{w.d}E{w.E}k{w.k}f{w.f}{'b' if w.backward else ''}")
-@pytest.mark.parametrize("path", [binding.GEMM_SCALAR, binding.GEMM_AUTO], ids=["scalar", "auto"])
+@pytest.mark.parametrize("path", [binding.GEMM_SCALAR, binding.GEMM_AUTO, binding.GEMM_TENSOR_TN],
+                         ids=["scalar", "auto", "tokens_on_n"])
 def test_small_layers_match_oracle(w, path):
+    if path == binding.GEMM_TENSOR_TN and (w.d % 64 or w.f % 64):
+        with pytest.raises(binding.MopError) as e:      # a forced tensor-core schedule refuses odd shapes
+            binding.context_for(w, gemm_path=path)
+        assert e.value.code == 6
+        return
     check_layer(w, path)
 
 
-@pytest.mark.parametrize("path", [binding.GEMM_TENSOR_2CTA, binding.GEMM_TENSOR_MIXED], ids=["2cta", "mixed"])
+@pytest.mark.parametrize("path", [binding.GEMM_TENSOR_2CTA, binding.GEMM_TENSOR_MIXED, binding.GEMM_TENSOR_TN],
+                         ids=["2cta", "mixed", "tokens_on_n"])
 def test_two_cta_schedules_match_oracle_and_the_one_cta_kernel(path):
     w = synth.small("c2_mid", T=1500, d=256, E=6, k=2, f=320, backward=True, seed=21)   # 500 rows per expert
     _, buf = check_layer(w, path)
