@@ -30,7 +30,7 @@ if str(ROOT) not in sys.path:
 import numpy as np
 import torch
 
-from paper_2607_01844_b200 import synth
+from paper_2607_01844_b200 import launch, synth
 
 # fallback denominators if MEASURED_PEAKS.json is absent (an earlier measurement on this machine)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -224,20 +224,13 @@ def main():
     args.warmup = max(3, args.warmup or 3)
 
     from paper_2607_01844_b200 import binding
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = launch.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
+    launch.init("nccl", dev)
+    barrier = launch.barrier
 
     inp = synth.make_inputs(w, dev)
     ctx = binding.context_for(w, device=local, host_io=not args.no_e2e, gemm_path=args.gemm_path)
@@ -269,12 +262,9 @@ def main():
     prof = binding.mop_profile_read(ctx, stream)
     binding.mop_profile_enable(ctx, False)
     binding.mop_poll(ctx, stream)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = launch.max_over_ranks(ms, dev)
     ms_step = ms / args.steps
-    value = world * flops_per_step(w) / (ms_step * 1e-3) / 1e12
+    value = launch.job_throughput(flops_per_step(w), ms_step, world) / 1e12
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -312,12 +302,9 @@ def main():
         e1.record(stream)
         torch.cuda.synchronize(); barrier()
         ems = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ems], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
+        ems = launch.max_over_ranks(ems, dev)
         assert torch.equal(Yh, buf.Y.cpu()), "host entry point and device path disagree"
-        e2e = {"value": world * flops_per_step(w) / (ems / n_e2e * 1e-3) / 1e12, "unit": "TFLOP/s",
+        e2e = {"value": launch.job_throughput(flops_per_step(w), ems / n_e2e, world) / 1e12, "unit": "TFLOP/s",
                "ms_per_step": ems / n_e2e, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank != 0:

@@ -36,6 +36,8 @@ struct mop_ctx {
     bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
     int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
     float *hgate, *hdgate;
+    cudaStream_t copy_stream;            // host-buffer entry points: copies that overlap the kernels
+    cudaEvent_t ev_in, ev_mid, ev_out;
     TcPlan plan;
     Profiler prof;
 };
@@ -246,6 +248,14 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         }
     }
     if (cudaMemset(c->status, 0, 256) != cudaSuccess) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
+    if (shape->host_io) {
+        if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_mid, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming) != cudaSuccess) {
+            cudaFree(c->ws); delete c; return MOP_ERR_CUDA;
+        }
+    }
     if (c->tensor_ok) {
         st = tc_plan_init(&c->plan, *shape, c->sm_count, &c->prof);
         if (st == MOP_OK) st = tc2_init();
@@ -272,6 +282,10 @@ void mop_destroy(mop_ctx* c) {
     if (c->prof.ev) {
         for (int i = 0; i < 2 * Profiler::MAX_REC; ++i) cudaEventDestroy(c->prof.ev[i]);
         delete[] c->prof.ev;
+    }
+    if (c->s.host_io) {
+        cudaStreamDestroy(c->copy_stream);
+        cudaEventDestroy(c->ev_in); cudaEventDestroy(c->ev_mid); cudaEventDestroy(c->ev_out);
     }
     cudaFree(c->ws);
     delete c;
@@ -498,9 +512,17 @@ mop_status step_host(mop_ctx* c, const void* x_host, const void* dY_host, const 
     if (!guard.ok) return MOP_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t M = (size_t)s.T * s.k, xb = (size_t)s.T * s.d * 2;
+    // Copies that the kernels do not wait for run on the context's copy stream: dY comes in while the
+    // forward runs, Y (and the routing) goes out while the backward runs.
+    cudaStream_t cs = c->copy_stream;
     if (s.T > 0) {
         CUDA_OK(cudaMemcpyAsync(c->hx, x_host, xb, cudaMemcpyHostToDevice, st));
-        if (bwd) CUDA_OK(cudaMemcpyAsync(c->hdY, dY_host, xb, cudaMemcpyHostToDevice, st));
+        if (bwd) {
+            CUDA_OK(cudaEventRecord(c->ev_in, st));            // orders the copy stream after earlier work on st
+            CUDA_OK(cudaStreamWaitEvent(cs, c->ev_in, 0));
+            CUDA_OK(cudaMemcpyAsync(c->hdY, dY_host, xb, cudaMemcpyHostToDevice, cs));
+            CUDA_OK(cudaEventRecord(c->ev_in, cs));
+        }
     }
     mop_status r;
     if ((r = mop_moe_route(c, c->hx, W_r, bias, c->hidx, c->hgate, nullptr, stream)) != MOP_OK) return r;
@@ -510,19 +532,27 @@ mop_status step_host(mop_ctx* c, const void* x_host, const void* dY_host, const 
                                     bwd ? c->hG : nullptr, bwd ? c->hU : nullptr, c->hH, c->hYp, stream)) != MOP_OK)
         return r;
     if ((r = mop_moe_combine(c, c->hYp, c->hperm, c->hY, stream)) != MOP_OK) return r;
+    if (s.T > 0) {
+        cudaStream_t os = bwd ? cs : st;                       // forward only: nothing to overlap with
+        if (bwd) {
+            CUDA_OK(cudaEventRecord(c->ev_mid, st));
+            CUDA_OK(cudaStreamWaitEvent(cs, c->ev_mid, 0));
+        }
+        CUDA_OK(cudaMemcpyAsync(Y_host, c->hY, xb, cudaMemcpyDeviceToHost, os));
+        if (idx_host) CUDA_OK(cudaMemcpyAsync(idx_host, c->hidx, M * 4, cudaMemcpyDeviceToHost, os));
+        if (gate_host) CUDA_OK(cudaMemcpyAsync(gate_host, c->hgate, M * 4, cudaMemcpyDeviceToHost, os));
+        if (bwd) CUDA_OK(cudaEventRecord(c->ev_out, cs));
+    }
     if (bwd) {
+        if (s.T > 0) CUDA_OK(cudaStreamWaitEvent(st, c->ev_in, 0));   // dY has arrived
         if ((r = mop_moe_expert_ffn_bwd(c, c->hdY, c->hXp, c->hG, c->hU, c->hH, c->hoffsets, c->hperm, c->hsrc,
                                         c->hgate, W_gate, W_up, W_down, c->hdX, dW_gate, dW_up, dW_down, c->hdgate,
                                         stream)) != MOP_OK)
             return r;
-    }
-    if (s.T > 0) {
-        CUDA_OK(cudaMemcpyAsync(Y_host, c->hY, xb, cudaMemcpyDeviceToHost, st));
-        if (idx_host) CUDA_OK(cudaMemcpyAsync(idx_host, c->hidx, M * 4, cudaMemcpyDeviceToHost, st));
-        if (gate_host) CUDA_OK(cudaMemcpyAsync(gate_host, c->hgate, M * 4, cudaMemcpyDeviceToHost, st));
-        if (bwd) {
+        if (s.T > 0) {
             CUDA_OK(cudaMemcpyAsync(dX_host, c->hdX, xb, cudaMemcpyDeviceToHost, st));
             if (dgate_host) CUDA_OK(cudaMemcpyAsync(dgate_host, c->hdgate, M * 4, cudaMemcpyDeviceToHost, st));
+            CUDA_OK(cudaStreamWaitEvent(st, c->ev_out, 0));     // st completes only after the Y copy
         }
     }
     CUDA_OK(cudaStreamSynchronize(st));
