@@ -44,10 +44,10 @@ struct TcTraits {
     static constexpr int N_PER_TILE = DUAL_B ? 128 : 256;             // output columns per tensor per tile
     // Weight gradients have a short K loop (the expert's rows) and a 128 KiB fp32 tile to write, so
     // they run eight epilogue warps (two per TMEM lane quarter, 128 columns each).
-    static constexpr int STAGES = 4;
+    static constexpr int STAGES = RAGGED_K ? 3 : 4;
     static constexpr int EPI_WARPS = RAGGED_K ? 8 : 4;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
-    static constexpr int STORE_BYTES = RAGGED_K ? EPI_WARPS * 4096 : 0;   // 32x32 fp32 transpose buffer per warp
+    static constexpr int STORE_BYTES = RAGGED_K ? 4 * 16384 : 0;   // two 128-row x 32-column fp32 store boxes per half
     static constexpr int SMEM_BYTES = STAGES * TC_STAGE_BYTES + 1024 /*align*/ + TC_BAR_BYTES + STORE_BYTES;
 };
 
@@ -503,6 +503,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 belong to this warp
         const int r = quarter * 32 + lane;       // row of the tile owned by this thread
         const int half = (warp - 2) >> 2;        // eight-warp epilogue: columns [128*half, 128*half + 128)
+        int sbuf = 0;                            // weight gradients: store box in use
         int it = 0;
         TileInfo nxt = decode_tile<KIND>(args, min((int)blockIdx.x, max(total_tiles - 1, 0)));
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
@@ -536,14 +537,15 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             if constexpr (!Tr::RAGGED_K) {
                 tc_epilogue_rows<KIND>(args, taddr, row_ok, grow, n0, ti.nt);
             } else {
-                // Weight-gradient tile: each warp transposes 32 rows x 32 fp32 columns through shared
-                // memory (128-byte rows, 16-byte chunks XOR-swizzled by row: conflict-free both ways)
-                // so that its global stores are whole 128-byte lines: 8 lanes per row, 4 rows per
-                // instruction.  Rows >= Mfix and columns >= N are not written.
-                float* sb = reinterpret_cast<float*>(smem + TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + (warp - 2) * 4096);
-                float* outp = (Tr::DUAL_B && half) ? args.outf1 : args.ep.outf;
-                const int row_base = ti.m0 + quarter * 32;
-                const size_t obase = ((size_t)ti.e * args.Mfix + row_base) * args.N;
+                // Weight-gradient tile: the four warps of a column half stage 128 rows x 32 fp32 columns
+                // in shared memory (128-byte rows, 16-byte chunks XOR-swizzled by row: the layout of a
+                // 128B-swizzle tensor map, conflict-free for one-row-per-lane writes) and one thread hands
+                // the 16 KiB box to TMA, which writes whole 128-byte lines and clips rows >= Mfix and
+                // columns >= N.  Only the box writes use the load/store pipe.  Two boxes per half.
+                uint8_t* gbase = smem + TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + half * 32768;
+                const CUtensorMap* mo = (Tr::DUAL_B && half) ? &tmO1 : &tmO0;
+                const bool issuer = (quarter == 0 && lane == 0);
+                const int gbar = 1 + half;               // named barrier of this half's 128 threads
                 float acc_b[32];
 #pragma unroll 1
                 for (int c = half * 128; c < half * 128 + 128; c += 64) {
@@ -552,29 +554,28 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                     tmem_ld_wait(acc, acc_b);
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        __syncwarp();
+                        uint8_t* box = gbase + (sbuf & 1) * 16384;
+                        if (issuer) tma_store_wait_read<1>();     // the box staged two steps ago has been read
+                        asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
+                        uint8_t* rowp = box + (quarter * 32 + lane) * 128;
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             const float4 v = h ? make_float4(acc_b[4 * j], acc_b[4 * j + 1], acc_b[4 * j + 2], acc_b[4 * j + 3])
                                                : make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
-                            *reinterpret_cast<float4*>(sb + lane * 32 + ((j ^ (lane & 7)) << 2)) = v;
+                            *reinterpret_cast<float4*>(rowp + ((j ^ (lane & 7)) << 4)) = v;
                         }
-                        __syncwarp();
-                        const int col = c + 32 * h;
-                        const int gcol = n0 + (Tr::DUAL_B ? (col & 127) : col) + (lane & 7) * 4;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int rr = 4 * i + (lane >> 3);
-                            float4 v = *reinterpret_cast<const float4*>(sb + rr * 32 + (((lane & 7) ^ (rr & 7)) << 2));
-                            if (row_base + rr < args.Mfix && gcol < args.N) {
-                                float4* dst = reinterpret_cast<float4*>(outp + obase + (size_t)rr * args.N + gcol);
-                                if (args.ep.accumulate) {
-                                    const float4 o = *dst;
-                                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                                }
-                                *dst = v;
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
+                        if (issuer) {
+                            const int col = c + 32 * h;
+                            const int gcol = n0 + (Tr::DUAL_B ? (col & 127) : col);
+                            if (gcol < args.N) {
+                                if (args.ep.accumulate) tma_reduce_add_3d(mo, smem_u32(box), gcol, ti.m0, ti.e);
+                                else tma_store_3d(mo, smem_u32(box), gcol, ti.m0, ti.e);
                             }
+                            tma_store_commit();
                         }
+                        ++sbuf;
                     }
                 }
             }
@@ -583,6 +584,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             if (lane == 0) mbar_arrive(tempty_bar(buf));
             ++it;
         }
+        if (Tr::RAGGED_K && quarter == 0 && lane == 0) tma_store_wait_all();   // boxes read before the CTA exits
+        (void)sbuf;
     }
 
     // ------------------------------------------------------------------------- teardown
@@ -709,12 +712,12 @@ inline bool tc_map_chunked_3d(const TcPlan* p, CUtensorMap* m, const void* base,
                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 3-D map over a dense [E, rows, cols] fp32 tensor for stores; box = {32 cols, 32 rows, 1}.
+// 3-D map over a dense [E, rows, cols] fp32 tensor for stores; box = {32 cols, 128 rows, 1}.
 inline bool tc_map_out_f32(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows,
                            uint64_t cols) {
     const cuuint64_t dims[3] = {cols, rows, E};
     const cuuint64_t strides[2] = {cols * 4, rows * cols * 4};
-    const cuuint32_t box[3] = {32, 32, 1};
+    const cuuint32_t box[3] = {32, 128, 1};
     const cuuint32_t es[3] = {1, 1, 1};
     return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base),
                                                      dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
