@@ -238,3 +238,41 @@ def ffn_bwd_experts(x, dY, idx, gate, Wg, Wu, Wd, experts, *, fp64=False, declar
                 _p(dWg), _p(dWu), _p(dWd))
     _check(rc, name)
     return dWg, dWu, dWd
+
+
+# ----------------------------------------------------------------------------- router backward
+def route_bwd(x_bits, W_r, bias, k, score_fn, bias_mode, idx, dgate):
+    """Backward of the router's gate computation with the selection held fixed (plain numpy, fp64).
+
+    The gates of a token are g_j = s_j / sum_l s_l over its k selected experts, with s = softmax
+    over all E of the logits (softmax router; the common denominator cancels, so g is a softmax
+    over the selected logits) or s = sigmoid(logit) (sigmoid router); logit = z (+ bias when the
+    bias enters before the score), z = x W_r.  Given dL/dgate this returns
+        dz     [T,E]  (non-zero only at the selected experts),
+        dW_r   [d,E] = x^T dz,   dX [T,d] = dz W_r^T,   dbias [E] (zero unless the bias is pre-logit).
+    A bias added after the score only steers the selection and receives no gradient.
+    """
+    x = bf16_bits_to_f64(x_bits)
+    W = np.asarray(W_r, np.float64)
+    T, d = x.shape
+    E = W.shape[1]
+    idx = np.asarray(idx, np.int64)
+    dg = np.asarray(dgate, np.float64)
+    zz = x @ W
+    if bias_mode == BIAS_PRE_LOGIT:
+        zz = zz + np.asarray(bias, np.float64)[None, :]
+    zs = np.take_along_axis(zz, idx, 1)                     # logits of the selected experts [T,k]
+    if score_fn == SCORE_SOFTMAX:
+        p = np.exp(zs - zs.max(1, keepdims=True))
+        g = p / p.sum(1, keepdims=True)
+        dzs = g * (dg - (g * dg).sum(1, keepdims=True))
+    else:
+        s = 1.0 / (1.0 + np.exp(-zs))
+        S = s.sum(1, keepdims=True)
+        g = s / S
+        ds = (dg - (g * dg).sum(1, keepdims=True)) / S
+        dzs = ds * s * (1.0 - s)
+    dz = np.zeros((T, E))
+    np.put_along_axis(dz, idx, dzs, 1)
+    dbias = dz.sum(0) if bias_mode == BIAS_PRE_LOGIT else np.zeros(E)
+    return dz, x.T @ dz, dz @ W.T, dbias

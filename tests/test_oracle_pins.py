@@ -337,3 +337,69 @@ def test_declared_rounding_mode_stays_close_to_exact_mode():
     # outputs declared bf16 are representable in bf16
     for b in de[:2]:
         assert np.array_equal(oracle.bf16_bits_to_f32(synth.bits(torch.from_numpy(b).to(torch.bfloat16))), b)
+
+
+# ------------------------------------------------------------------------------ router backward
+@pytest.mark.parametrize("score_fn,bias_mode", [(0, 0), (0, 2), (1, 0), (1, 1), (1, 2)])
+def test_router_backward_matches_automatic_differentiation_of_the_long_form(score_fn, bias_mode):
+    """The oracle uses the closed form on the selected logits; autodiff differentiates the long
+    form (scores over ALL experts, then renormalisation over the selected ones)."""
+    rng = np.random.default_rng(20 + score_fn * 3 + bias_mode)
+    T, d, E, k = 9, 12, 7, 3
+    x = _rand_bits(rng, (T, d))
+    Wr = (rng.standard_normal((d, E)) * 0.4).astype(np.float32)
+    b = (rng.standard_normal(E) * 0.1).astype(np.float32) if bias_mode else None
+    idx, gate = oracle.route(x, Wr, b, k, score_fn, bias_mode)
+    dgate = rng.standard_normal((T, k))
+    dz, dWr, dX, db = oracle.route_bwd(x, Wr, b, k, score_fn, bias_mode, idx, dgate)
+
+    tx = torch.tensor(oracle.bf16_bits_to_f64(x), requires_grad=True)
+    tW = torch.tensor(Wr.astype(np.float64), requires_grad=True)
+    tb = torch.tensor(b.astype(np.float64), requires_grad=True) if bias_mode else None
+    z = tx @ tW
+    if bias_mode == 2:
+        z = z + tb
+    s = torch.softmax(z, 1) if score_fn == 0 else torch.sigmoid(z)
+    sel = torch.gather(s, 1, torch.from_numpy(idx.astype(np.int64)))
+    g = sel / sel.sum(1, keepdim=True)
+    assert np.max(np.abs(g.detach().numpy() - gate)) < 1e-6          # same forward as the router
+    (g * torch.from_numpy(dgate)).sum().backward()
+    assert np.max(np.abs(dWr - tW.grad.numpy())) < 1e-12
+    assert np.max(np.abs(dX - tx.grad.numpy())) < 1e-12
+    if bias_mode == 2:
+        assert np.max(np.abs(db - tb.grad.numpy())) < 1e-12
+    else:
+        assert np.all(db == 0)
+        if bias_mode == 1:
+            assert tb.grad is None                                       # selection only: no gradient
+    # dz is supported on the selected experts and sums to zero per token for softmax
+    mask = np.zeros((T, E), bool)
+    np.put_along_axis(mask, idx.astype(np.int64), True, 1)
+    assert np.all(dz[~mask] == 0)
+    if score_fn == 0:
+        assert np.max(np.abs(dz.sum(1))) < 1e-12
+
+
+def test_router_backward_central_differences():
+    rng = np.random.default_rng(31)
+    T, d, E, k = 5, 8, 6, 2
+    x = _rand_bits(rng, (T, d))
+    Wr = (rng.standard_normal((d, E)) * 0.4).astype(np.float32)
+    idx, _ = oracle.route(x, Wr, None, k, 1, 0)
+    dgate = rng.standard_normal((T, k))
+    _, dWr, _, _ = oracle.route_bwd(x, Wr, None, k, 1, 0, idx, dgate)
+    xf = oracle.bf16_bits_to_f64(x)
+
+    def loss(W):
+        z = np.take_along_axis(xf @ W, idx.astype(np.int64), 1)
+        s = 1 / (1 + np.exp(-z))
+        return float(((s / s.sum(1, keepdims=True)) * dgate).sum())
+
+    W0 = Wr.astype(np.float64)
+    for _ in range(10):
+        i, e = rng.integers(0, d), rng.integers(0, E)
+        Wp, Wm = W0.copy(), W0.copy()
+        Wp[i, e] += 1e-6
+        Wm[i, e] -= 1e-6
+        fd = (loss(Wp) - loss(Wm)) / 2e-6
+        assert abs(fd - dWr[i, e]) <= 1e-6 * max(1.0, abs(dWr[i, e]))
