@@ -64,6 +64,8 @@ def kernel_work(w, counts):
     return {
         "route_score": (2 * T * d * E, T * d * 2 + d * E * 4 + T * E * 4),
         "route_select": (0, T * E * 4 + T * k * 8),
+        "route_bwd_dwr": (2 * M * d, M * d * 2 + M * 4 + d * E * 4),
+        "route_bwd_dx": (2 * M * d, 2 * T * d * 2 + T * k * 8 + d * E * 4),
         "permute_scatter_rows": (0, T * d * 2 + M * d * 2 + M * 4),
         "dy_scatter_rows": (0, T * d * 2 + M * d * 2 + M * 4),
         "combine_rows": (0, M * d * 2 + T * d * 2 + M * 4),
@@ -211,6 +213,8 @@ def main():
                     help="T,d,E,k,f overriding the named workload's sizes (same distributions): small cases for "
                          "profiler captures")
     ap.add_argument("--gemm-path", type=int, default=0, help="mop_gemm_path (0 = library default)")
+    ap.add_argument("--with-router-bwd", action="store_true",
+                    help="also run the router backward (dgate -> dW_r, dX) in every step of a fwd+bwd workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -240,10 +244,26 @@ def main():
     buf = binding.LayerBuffers(w, device=dev)
     stream = torch.cuda.current_stream()
 
+    rbwd = args.with_router_bwd and w.backward
+    if rbwd:
+        logits = torch.empty((w.T, w.E), dtype=torch.float32, device=dev)
+        dW_r = torch.empty((w.d, w.E), dtype=torch.float32, device=dev)
+
     def step():
-        binding.forward(ctx, inp, buf, stream)
+        if rbwd:   # the router keeps its logits for the backward
+            binding.mop_moe_route(ctx, inp["x"], inp["W_r"], inp["bias"], buf.idx, buf.gate, logits, stream)
+            binding.mop_moe_permute(ctx, inp["x"], buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, buf.Xp,
+                                    stream)
+            binding.mop_moe_expert_ffn_fwd(ctx, buf.Xp, buf.offsets, buf.row_src, buf.gate, inp["W_gate"], inp["W_up"],
+                                           inp["W_down"], buf.G, buf.U, buf.H, buf.Yp, stream)
+            binding.mop_moe_combine(ctx, buf.Yp, buf.perm_row, buf.Y, stream)
+        else:
+            binding.forward(ctx, inp, buf, stream)
         if w.backward:
             binding.backward(ctx, inp, buf, stream)
+        if rbwd:
+            binding.mop_moe_route_bwd(ctx, logits, inp["bias"], buf.idx, buf.gate, buf.dgate, buf.Xp, buf.offsets,
+                                      buf.perm_row, inp["W_r"], dW_r, None, buf.dX, stream)
 
     for _ in range(args.warmup):
         step()

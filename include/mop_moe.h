@@ -137,6 +137,23 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* ctx, const void* dY, const void* Xp, 
                                   const void* W_up, const void* W_down, void* dX, float* dW_gate, float* dW_up,
                                   float* dW_down, float* dgate, void* stream);
 
+/* Router backward with the selection held fixed (Section 2.1's router, differentiated through the
+ * gate renormalisation and the score function; the step on either side of the expert path).
+ *   softmax:  dz_j = g_j (dgate_j - sum_l g_l dgate_l)
+ *   sigmoid:  dz_j = (dgate_j - sum_l g_l dgate_l) / S * s_j (1 - s_j),  s = sigmoid(logit), S = sum_l s_l
+ * over a token's k selected experts (dz = 0 elsewhere), then
+ *   dW_r = x^T dz,   dX += dz W_r^T   (added to the expert-path gradient already in dX),
+ *   dbias = column sums of dz for MOP_BIAS_PRE_LOGIT (a post-score bias only steers the selection).
+ * logits [T,E] f32 as returned by mop_moe_route (logits_opt); topk_idx, topk_gate [T,k];
+ * dgate [T,k] f32 (from mop_moe_expert_ffn_bwd); Xp [T*k,d] bf16, offsets [E+1], perm_row [T*k]
+ * from mop_moe_permute; W_r [d,E] f32; bias as in mop_moe_route;
+ * dW_r [d,E] f32 out; dbias_opt [E] f32 out or NULL; dX [T,d] bf16 in/out.
+ * Needs a context created with with_backward = 1. */
+mop_status mop_moe_route_bwd(mop_ctx* ctx, const float* logits, const float* bias, const int32_t* topk_idx,
+                             const float* topk_gate, const float* dgate, const void* Xp, const int32_t* offsets,
+                             const int32_t* perm_row, const float* W_r, float* dW_r, float* dbias_opt, void* dX,
+                             void* stream);
+
 /* Whole forward with HOST buffers (pageable or pinned): copies x in, runs route, permute,
  * expert_ffn_fwd and combine on `stream`, copies Y, topk_idx and topk_gate back, and
  * synchronises.  Weights stay on the device (they are parameters, not step inputs).

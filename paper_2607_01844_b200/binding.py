@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_combine.argtypes = [_P] * 5
         L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 19
         L.mop_moe_forward_host.argtypes = [_P] * 11
+        L.mop_moe_route_bwd.argtypes = [_P] * 14
         L.mop_moe_train_step_host.argtypes = [_P] * 15
         L.mop_moe_permute_static.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 4 + [_P] * 8
         L.mop_profile_enable.argtypes = [_P, ctypes.c_int]
@@ -151,6 +152,14 @@ def mop_moe_expert_ffn_bwd(ctx, dY, Xp, G_save, U_save, H, offsets, perm_row, ro
                                         _ptr(offsets), _ptr(perm_row), _ptr(row_src), _ptr(topk_gate), _ptr(W_gate),
                                         _ptr(W_up), _ptr(W_down), _ptr(dX), _ptr(dW_gate), _ptr(dW_up), _ptr(dW_down),
                                         _ptr(dgate), _stream(stream)))
+
+
+def mop_moe_route_bwd(ctx, logits, bias, topk_idx, topk_gate, dgate, Xp, offsets, perm_row, W_r, dW_r, dbias, dX,
+                      stream=None):
+    _check("mop_moe_route_bwd",
+           lib().mop_moe_route_bwd(ctx.handle, _ptr(logits), _ptr(bias), _ptr(topk_idx), _ptr(topk_gate), _ptr(dgate),
+                                   _ptr(Xp), _ptr(offsets), _ptr(perm_row), _ptr(W_r), _ptr(dW_r), _ptr(dbias),
+                                   _ptr(dX), _stream(stream)))
 
 
 def mop_moe_forward_host(ctx, x_host, W_r, bias, W_gate, W_up, W_down, Y_host, idx_host=None, gate_host=None,

@@ -32,6 +32,7 @@ struct mop_ctx {
     int32_t* status;     // device status word
     float* part;         // [ntile_max, M] partial dot products for dgate
     bf16 *dYp, *dG, *dU, *gH, *dXp;  // backward intermediates
+    float *dz_sel, *dz_row, *wrT;    // router backward: dz per assignment / per permuted row; W_r^T [E,d]
     // host-buffer entry point scratch
     bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
     int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
@@ -47,7 +48,7 @@ namespace {
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 struct Layout {
-    size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp;
+    size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
     size_t hG, hU, hdY, hdX, hdgate;
     size_t total;
@@ -72,6 +73,9 @@ Layout make_layout(const mop_moe_shape& s) {
         L.dU = take(M * f * 2);
         L.gH = take(M * f * 2);
         L.dXp = take(M * d * 2);
+        L.dz_sel = take(M * 4 + 16);
+        L.dz_row = take(M * 4 + 16);
+        L.wrT = take(d * E * 4);
     }
     if (s.host_io) {
         L.hx = take(T * d * 2);
@@ -226,6 +230,9 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         c->dU = reinterpret_cast<bf16*>(w + L.dU);
         c->gH = reinterpret_cast<bf16*>(w + L.gH);
         c->dXp = reinterpret_cast<bf16*>(w + L.dXp);
+        c->dz_sel = reinterpret_cast<float*>(w + L.dz_sel);
+        c->dz_row = reinterpret_cast<float*>(w + L.dz_row);
+        c->wrT = reinterpret_cast<float*>(w + L.wrT);
     }
     if (shape->host_io) {
         c->hx = reinterpret_cast<bf16*>(w + L.hx);
@@ -499,6 +506,44 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
            dgate_reduce_kernel<<<ceil_div(M, 256), 256, 0, st>>>(c->part, perm_row, dgate, M, ntile_part));
     if ((r = after_launch(c)) != MOP_OK) return r;
     return mop_moe_combine(c, c->dXp, perm_row, dX, stream);
+}
+
+mop_status mop_moe_route_bwd(mop_ctx* c, const float* logits, const float* bias, const int32_t* topk_idx,
+                             const float* topk_gate, const float* dgate, const void* Xp, const int32_t* offsets,
+                             const int32_t* perm_row, const float* W_r, float* dW_r, float* dbias_opt, void* dX,
+                             void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (!c->s.with_backward) return MOP_ERR_UNSUPPORTED;
+    REQ_PTR_T(logits); REQ_PTR_T(topk_idx); REQ_PTR_T(topk_gate); REQ_PTR_T(dgate); REQ_PTR_T(Xp); REQ_PTR(offsets);
+    REQ_PTR_T(perm_row); REQ_PTR(W_r); REQ_PTR(dW_r); REQ_PTR_T(dX);
+    if ((c->s.bias_mode != MOP_BIAS_NONE) != (bias != nullptr)) return MOP_ERR_INVALID_ARG;
+    if (dbias_opt && !aligned16(dbias_opt)) return MOP_ERR_ALIGN;
+    const mop_moe_shape& s = c->s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    mop_status r;
+    if (s.T > 0) {
+        LAUNCH(c, "route_bwd_dz", st,
+               route_bwd_dz_kernel<<<ceil_div(s.T, 8), 256, 0, st>>>(logits, bias, topk_idx, topk_gate, dgate, perm_row,
+                                                                     c->dz_sel, c->dz_row, s.T, s.E, s.k, s.score_fn,
+                                                                     s.bias_mode));
+        if ((r = after_launch(c)) != MOP_OK) return r;
+    }
+    dim3 gw(ceil_div(s.d, 1024), s.E);
+    float* db = (dbias_opt && s.bias_mode == MOP_BIAS_PRE_LOGIT) ? dbias_opt : nullptr;
+    if (dbias_opt && !db) CUDA_OK(cudaMemsetAsync(dbias_opt, 0, (size_t)s.E * 4, st));
+    LAUNCH(c, "route_bwd_dwr", st,
+           route_bwd_dwr_kernel<<<gw, 128, 0, st>>>(static_cast<const bf16*>(Xp), c->dz_row, offsets, dW_r, db, s.d, s.E));
+    if ((r = after_launch(c)) != MOP_OK) return r;
+    if (s.T == 0) return MOP_OK;
+    dim3 gt(ceil_div(s.E, 32), ceil_div(s.d, 32));
+    LAUNCH(c, "route_bwd_wrT", st, transpose_f32_kernel<<<gt, 256, 0, st>>>(W_r, c->wrT, s.d, s.E));
+    if ((r = after_launch(c)) != MOP_OK) return r;
+    LAUNCH(c, "route_bwd_dx", st,
+           route_bwd_dx_kernel<<<s.T, 256, 0, st>>>(c->wrT, topk_idx, c->dz_sel, static_cast<bf16*>(dX), s.T, s.d, s.E,
+                                                    s.k));
+    return after_launch(c);
 }
 
 namespace {

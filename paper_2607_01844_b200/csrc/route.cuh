@@ -292,4 +292,139 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) route_select_kernel(const floa
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Router backward (selection held fixed).  With g_j = s_j / sum_l s_l over a token's k selected
+// experts (s = softmax over all E, whose common denominator cancels, or s = sigmoid):
+//   softmax:  dz_j = g_j (dgate_j - sum_l g_l dgate_l)
+//   sigmoid:  dz_j = (dgate_j - sum_l g_l dgate_l) / S * s_j (1 - s_j),   S = sum_l s_l
+// dz is zero at every expert that was not selected.  Then dW_r = x^T dz, dX += dz W_r^T and, for a
+// bias added before the score, dbias = column sums of dz.
+// ---------------------------------------------------------------------------------------------
+
+// One warp per token: lane j < k owns the j-th selected expert.  Writes dz per assignment and, in
+// expert-contiguous row order (row = perm_row[assignment]), the copy that the dW_r kernel reads.
+__global__ void __launch_bounds__(256) route_bwd_dz_kernel(const float* __restrict__ logits,
+                                                           const float* __restrict__ bias,
+                                                           const int32_t* __restrict__ idx,
+                                                           const float* __restrict__ gate,
+                                                           const float* __restrict__ dgate,
+                                                           const int32_t* __restrict__ perm_row,
+                                                           float* __restrict__ dz_sel, float* __restrict__ dz_row,
+                                                           int T, int E, int k, int score_fn, int bias_mode) {
+    const int lane = threadIdx.x % 32;
+    const int t = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    if (t >= T) return;
+    const bool act = lane < k;
+    const size_t a = (size_t)t * k + lane;
+    float g = 0.0f, dg = 0.0f, zz = 0.0f;
+    if (act) {
+        const int e = idx[a];
+        g = gate[a];
+        dg = dgate[a];
+        zz = logits[(size_t)t * E + e];
+        if (bias_mode == 2) zz += bias[e];
+    }
+    float dot = g * dg;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    float dz;
+    if (score_fn == 0) {
+        dz = g * (dg - dot);
+    } else {
+        const float s = act ? sigmoidf_acc(zz) : 0.0f;
+        float S = s;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) S += __shfl_xor_sync(0xffffffffu, S, off);
+        dz = (dg - dot) / S * s * (1.0f - s);
+    }
+    if (act) {
+        dz_sel[a] = dz;
+        const int32_t p = perm_row[a];
+        if (p >= 0) dz_row[p] = dz;
+    }
+}
+
+// dW_r[i,e] = sum over the rows p of expert e (ascending) of Xp[p,i] * dz_row[p].  Block (i-chunk, e):
+// 128 threads, eight columns i each (16-byte loads); Xp rows are read once, coalesced, two rows in
+// flight per thread.  Deterministic (no atomics).
+__global__ void __launch_bounds__(128) route_bwd_dwr_kernel(const bf16* __restrict__ Xp,
+                                                            const float* __restrict__ dz_row,
+                                                            const int32_t* __restrict__ offsets,
+                                                            float* __restrict__ dW_r, float* __restrict__ dbias,
+                                                            int d, int E) {
+    const int e = blockIdx.y;
+    const int i = (blockIdx.x * 128 + threadIdx.x) * 8;
+    const int p0 = offsets[e], p1 = offsets[e + 1];
+    if (i < d) {
+        float a[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) a[q] = 0.0f;
+        auto add = [&](const uint4& v, float w) {
+            a[0] = fmaf(bf16_lo(v.x), w, a[0]); a[1] = fmaf(bf16_hi(v.x), w, a[1]);
+            a[2] = fmaf(bf16_lo(v.y), w, a[2]); a[3] = fmaf(bf16_hi(v.y), w, a[3]);
+            a[4] = fmaf(bf16_lo(v.z), w, a[4]); a[5] = fmaf(bf16_hi(v.z), w, a[5]);
+            a[6] = fmaf(bf16_lo(v.w), w, a[6]); a[7] = fmaf(bf16_hi(v.w), w, a[7]);
+        };
+        int p = p0;
+        for (; p + 1 < p1; p += 2) {
+            const uint4 v0 = __ldcs(reinterpret_cast<const uint4*>(Xp + (size_t)p * d + i));
+            const uint4 v1 = __ldcs(reinterpret_cast<const uint4*>(Xp + (size_t)(p + 1) * d + i));
+            add(v0, dz_row[p]);
+            add(v1, dz_row[p + 1]);
+        }
+        if (p < p1) add(__ldcs(reinterpret_cast<const uint4*>(Xp + (size_t)p * d + i)), dz_row[p]);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) dW_r[(size_t)(i + q) * E + e] = a[q];
+    }
+    if (dbias && blockIdx.x == 0 && threadIdx.x == 0) {
+        float sb = 0.0f;
+        for (int p = p0; p < p1; ++p) sb += dz_row[p];
+        dbias[e] = sb;
+    }
+}
+
+// W_r^T [E,d] from W_r [d,E] (32 x 32 tiles through shared memory): gives the dX kernel contiguous rows.
+__global__ void __launch_bounds__(256) transpose_f32_kernel(const float* __restrict__ in, float* __restrict__ out,
+                                                            int rows, int cols) {
+    __shared__ float tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    for (int r = ty; r < 32; r += 8)
+        if (r0 + r < rows && c0 + tx < cols) tile[r][tx] = in[(size_t)(r0 + r) * cols + c0 + tx];
+    __syncthreads();
+    for (int c = ty; c < 32; c += 8)
+        if (c0 + c < cols && r0 + tx < rows) out[(size_t)(c0 + c) * rows + r0 + tx] = tile[tx][c];
+}
+
+// dX[t,:] += dz[t,:] W_r^T = sum_j dz[t,j] * W_r^T[e_j,:]: one CTA per token walks its k selected rows
+// of W_r^T (contiguous, L2-resident) four columns per thread; dX is read, updated in fp32 and rounded
+// back to bf16.  d is a multiple of 8.
+__global__ void __launch_bounds__(256) route_bwd_dx_kernel(const float* __restrict__ W_rT,
+                                                           const int32_t* __restrict__ idx,
+                                                           const float* __restrict__ dz_sel, bf16* __restrict__ dX,
+                                                           int T, int d, int E, int k) {
+    __shared__ int32_t es[32];
+    __shared__ float dzs[32];
+    const int t = blockIdx.x;
+    if (threadIdx.x < k) {
+        es[threadIdx.x] = idx[(size_t)t * k + threadIdx.x];
+        dzs[threadIdx.x] = dz_sel[(size_t)t * k + threadIdx.x];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x * 4; i < d; i += 256 * 4) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < k; ++j) {
+            const float4 w = *reinterpret_cast<const float4*>(W_rT + (size_t)es[j] * d + i);
+            const float s = dzs[j];
+            acc.x = fmaf(s, w.x, acc.x); acc.y = fmaf(s, w.y, acc.y);
+            acc.z = fmaf(s, w.z, acc.z); acc.w = fmaf(s, w.w, acc.w);
+        }
+        uint2* px = reinterpret_cast<uint2*>(dX + (size_t)t * d + i);
+        uint2 v = *px;
+        v.x = pack_bf16x2(bf16_lo(v.x) + acc.x, bf16_hi(v.x) + acc.y);
+        v.y = pack_bf16x2(bf16_lo(v.y) + acc.z, bf16_hi(v.y) + acc.w);
+        *px = v;
+    }
+}
+
 }  // namespace mop

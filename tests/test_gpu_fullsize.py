@@ -119,3 +119,33 @@ def test_full_size_sampled(name):
             for nm, got, a, b in zip(("dW_gate", "dW_up", "dW_down"), (buf.dW_gate, buf.dW_up, buf.dW_down), dW_e,
                                      dW_d):
                 print(name, e, q["rows"], nm, check_float(nm, got[e].cpu().numpy(), a[0], b[0], scale(b)))
+
+
+def test_full_size_router_backward():
+    """Router backward at config 5's T, d, E, k (the expert width plays no part in it)."""
+    w = synth.small("c5_train", f=64)
+    dev = torch.device("cuda")
+    x = synth._normal_bf16((w.T, w.d), 1.0, synth._gen(w.seed, 1, dev), dev)
+    W_r = torch.randn((w.d, w.E), generator=synth._gen(w.seed, 2, dev), device=dev) * 0.02
+    bias = torch.randn((w.E,), generator=synth._gen(w.seed, 6, dev), device=dev) * w.bias_std
+    ctx = binding.context_for(w)
+    buf = binding.LayerBuffers(w)
+    logits = torch.empty((w.T, w.E), dtype=torch.float32, device=dev)
+    binding.mop_moe_route(ctx, x, W_r, bias, buf.idx, buf.gate, logits)
+    binding.mop_moe_permute(ctx, x, buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, buf.Xp)
+    g = torch.Generator(device=dev).manual_seed(99)
+    dgate = torch.randn((w.T, w.k), generator=g, device=dev) * 100.0          # dgate rms is about 140 at this size
+    dX0 = torch.randn((w.T, w.d), generator=g, device=dev).to(torch.bfloat16)
+    dX = dX0.clone()
+    dWr = torch.empty((w.d, w.E), device=dev)
+    binding.mop_moe_route_bwd(ctx, logits, bias, buf.idx, buf.gate, dgate, buf.Xp, buf.offsets, buf.perm_row, W_r, dWr,
+                              None, dX)
+    torch.cuda.synchronize()
+    dz, dWr_ref, dXr_ref, _ = oracle.route_bwd(synth.bits(x), W_r.cpu().numpy(), bias.cpu().numpy(), w.k, w.score_fn,
+                                               w.bias_mode, buf.idx.cpu().numpy(), dgate.cpu().numpy())
+    r = np.linalg.norm(dWr.cpu().numpy() - dWr_ref) / np.linalg.norm(dWr_ref)
+    assert r < 1e-5, r
+    want = dX0.float().cpu().numpy().astype(np.float64) + dXr_ref
+    got = dX.float().cpu().numpy()
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) < 4e-3
+    assert np.max(np.abs(got - want)) <= 2.0 ** -8 * np.abs(want).max()

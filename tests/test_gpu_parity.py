@@ -196,3 +196,44 @@ def test_forward_host_entry_point_matches_device_path():
     binding.mop_moe_forward_host(ctx, xh, inp["W_r"], inp["bias"], inp["W_gate"], inp["W_up"], inp["W_down"], Yh, idxh,
                                  gh)
     assert torch.equal(Yh, buf.Y.cpu()) and torch.equal(idxh, buf.idx.cpu()) and torch.equal(gh, buf.gate.cpu())
+
+
+ROUTER_BWD = [
+    synth.small("c1_tiny", T=200, d=128, E=8, k=2, f=64, backward=True, seed=30),                       # softmax
+    synth.small("c3_trillion", T=300, d=192, E=40, k=8, f=64, backward=True, seed=31),                  # sigmoid + post bias
+    synth.small("c3_trillion", T=130, d=64, E=33, k=3, f=64, bias_mode=2, backward=True, seed=32),      # sigmoid, pre-logit bias
+    synth.small("c2_mid", T=257, d=72, E=12, k=12, f=64, bias_mode=2, bias_std=0.1, backward=True, seed=33),  # softmax, k = E
+]
+
+
+@pytest.mark.parametrize("w", ROUTER_BWD, ids=lambda w: f"{w.name}-T{w.T}d{w.d}E{w.E}k{w.k}s{w.score_fn}b{w.bias_mode}")
+def test_router_backward_matches_oracle(w):
+    host = synth.make_inputs(w, "cpu")
+    if w.bias_mode and host["bias"] is None:
+        host["bias"] = torch.randn(w.E) * 0.1
+    inp = to_dev(host)
+    ctx = binding.context_for(w)
+    buf = binding.LayerBuffers(w)
+    logits = torch.empty((w.T, w.E), dtype=torch.float32, device="cuda")
+    binding.mop_moe_route(ctx, inp["x"], inp["W_r"], inp["bias"], buf.idx, buf.gate, logits)
+    binding.mop_moe_permute(ctx, inp["x"], buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, buf.Xp)
+    g = torch.Generator().manual_seed(w.seed)
+    dgate = torch.randn((w.T, w.k), generator=g).cuda()
+    dX0 = (torch.randn((w.T, w.d), generator=g) * 0.5).to(torch.bfloat16).cuda()
+    dX = dX0.clone()
+    dWr = torch.full((w.d, w.E), 7.0, device="cuda")
+    dbias = torch.full((w.E,), 7.0, device="cuda")
+    binding.mop_moe_route_bwd(ctx, logits, inp["bias"], buf.idx, buf.gate, dgate, buf.Xp, buf.offsets, buf.perm_row,
+                              inp["W_r"], dWr, dbias, dX)
+    torch.cuda.synchronize()
+    bias = None if host["bias"] is None else host["bias"].numpy()
+    idx = buf.idx.cpu().numpy()
+    dz, dWr_ref, dXr_ref, db_ref = oracle.route_bwd(synth.bits(host["x"]), host["W_r"].numpy(), bias, w.k, w.score_fn,
+                                                    w.bias_mode, idx, dgate.cpu().numpy())
+    assert rel_fro(dWr.cpu().numpy(), dWr_ref) < 1e-5
+    assert np.max(np.abs(dbias.cpu().numpy() - db_ref)) <= 1e-5 * max(1.0, np.abs(db_ref).max())
+    # dX = bf16(dX_in + router part): one bf16 rounding of the sum
+    want = dX0.float().cpu().numpy().astype(np.float64) + dXr_ref
+    got = dX.float().cpu().numpy()
+    assert np.max(np.abs(got - want)) <= 2.0 ** -8 * np.maximum(1.0, np.abs(want)).max()
+    assert rel_fro(got, want) < 4e-3
