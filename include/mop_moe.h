@@ -65,7 +65,8 @@ typedef struct {
     int32_t T, d, E, k, f;
     int32_t score_fn;      /* mop_score_fn */
     int32_t bias_mode;     /* mop_bias_mode; POST_SCORE requires MOP_SCORE_SIGMOID */
-    int32_t with_backward; /* 1: the context also holds the backward's intermediates */
+    int32_t with_backward; /* 1: the context also holds the backward's intermediates; 2: and buffers to
+                              recompute G, U, H in the backward (activation checkpointing) */
     int32_t dw_accumulate; /* 0: dW is overwritten (empty experts get zeros); 1: dW += */
     int32_t gemm_path;     /* mop_gemm_path; AUTO = tensor cores when the shape allows */
     int32_t host_io;       /* 1: the context also holds the activations of mop_moe_forward_host */
@@ -130,7 +131,10 @@ mop_status mop_moe_combine(mop_ctx* ctx, const void* Yp, const int32_t* perm_row
  *   dW_gate[e] = Xp_e^T dG_e;  dW_up[e] = Xp_e^T dU_e;  dW_down[e] = (gate * H_e)^T dY_e
  * dY [T,d] bf16; Xp, G_save, U_save, H, offsets, perm_row, row_src, topk_gate, W_* as above;
  * dX [T,d] bf16 out; dW_gate, dW_up [E,d,f] f32 out; dW_down [E,f,d] f32 out;
- * dgate [T,k] f32 out.  Needs a context created with with_backward = 1. */
+ * dgate [T,k] f32 out.  Needs a context created with with_backward >= 1.
+ * Activation checkpointing (Section 3.1 lists it among the ways to cut transient activation memory):
+ * with G_save, U_save and H all NULL (context created with with_backward = 2) the forward may have
+ * run without the stash and the up-projection is recomputed here from Xp, bit for bit. */
 mop_status mop_moe_expert_ffn_bwd(mop_ctx* ctx, const void* dY, const void* Xp, const void* G_save,
                                   const void* U_save, const void* H, const int32_t* offsets, const int32_t* perm_row,
                                   const int32_t* row_src, const float* topk_gate, const void* W_gate,

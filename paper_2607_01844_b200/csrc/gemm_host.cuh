@@ -42,8 +42,21 @@ inline mop_status tc_rows_gemm(const TcPlan* p, const char* name, const char* na
     return MOP_OK;
 }
 
+inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
+                                  int* launches, bool with_down);
+
 inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
                              int* launches) {
+    return tc_ffn_fwd_impl(p, a, tiles, status, st, launches, true);
+}
+// Up-projection + SwiGLU alone (the backward's recomputation of G, U, H).
+inline mop_status tc_up_only(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
+                             int* launches) {
+    return tc_ffn_fwd_impl(p, a, tiles, status, st, launches, false);
+}
+
+inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
+                                  int* launches, bool with_down) {
     const mop_moe_shape& s = p->s;
     const uint64_t M = (uint64_t)s.T * s.k;
     mop_status r;
@@ -75,6 +88,7 @@ inline mop_status tc_ffn_fwd(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int3
         if ((r = tc_rows_gemm<TC_F1>(p, "gemm_up_swiglu", "gemm_up_swiglu_2cta", mXp, mXp, mWg, mWu, mWg, mWu, g, tiles, st, launches)) != MOP_OK)
             return r;
     }
+    if (!with_down) return MOP_OK;
     if (tn_f2) {
         if ((r = tn_down_gate(p, a, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), status, st)) != MOP_OK) return r;
         ++*launches;

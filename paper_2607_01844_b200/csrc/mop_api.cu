@@ -32,6 +32,7 @@ struct mop_ctx {
     int32_t* status;     // device status word
     float* part;         // [ntile_max, M] partial dot products for dgate
     bf16 *dYp, *dG, *dU, *gH, *dXp;  // backward intermediates
+    bf16 *rG, *rU, *rH;              // recompute-in-backward buffers (activation checkpointing)
     float *dz_sel, *dz_row, *wrT;    // router backward: dz per assignment / per permuted row; W_r^T [E,d]
     // host-buffer entry point scratch
     bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
@@ -48,7 +49,7 @@ namespace {
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 struct Layout {
-    size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT;
+    size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT, rG, rU, rH;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
     size_t hG, hU, hdY, hdX, hdgate;
     size_t total;
@@ -76,6 +77,11 @@ Layout make_layout(const mop_moe_shape& s) {
         L.dz_sel = take(M * 4 + 16);
         L.dz_row = take(M * 4 + 16);
         L.wrT = take(d * E * 4);
+        if (s.with_backward == 2) {
+            L.rG = take(M * f * 2);
+            L.rU = take(M * f * 2);
+            L.rH = take(M * f * 2);
+        }
     }
     if (s.host_io) {
         L.hx = take(T * d * 2);
@@ -233,6 +239,11 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         c->dz_sel = reinterpret_cast<float*>(w + L.dz_sel);
         c->dz_row = reinterpret_cast<float*>(w + L.dz_row);
         c->wrT = reinterpret_cast<float*>(w + L.wrT);
+        if (shape->with_backward == 2) {
+            c->rG = reinterpret_cast<bf16*>(w + L.rG);
+            c->rU = reinterpret_cast<bf16*>(w + L.rU);
+            c->rH = reinterpret_cast<bf16*>(w + L.rH);
+        }
     }
     if (shape->host_io) {
         c->hx = reinterpret_cast<bf16*>(w + L.hx);
@@ -387,6 +398,34 @@ mop_status mop_moe_combine(mop_ctx* c, const void* Yp, const int32_t* perm_row, 
     return after_launch(c);
 }
 
+namespace {
+// G, U, H = SwiGLU up-projection of the permuted rows (the first half of the forward; also the
+// recomputation step of the backward).  Tensor-core or scalar path as the context was created.
+mop_status up_projection(mop_ctx* c, const void* Xp, const int32_t* offsets, const void* W_gate, const void* W_up,
+                         void* G_save, void* U_save, void* H, cudaStream_t st) {
+    const mop_moe_shape& s = c->s;
+    const int M = s.T * s.k;
+    if (use_tensor(c)) {
+        TcFwdArgs a{};
+        a.Xp = static_cast<const bf16*>(Xp); a.offsets = offsets;
+        a.W_gate = static_cast<const bf16*>(W_gate); a.W_up = static_cast<const bf16*>(W_up);
+        a.G_save = static_cast<bf16*>(G_save); a.U_save = static_cast<bf16*>(U_save); a.H = static_cast<bf16*>(H);
+        int n = 0;
+        mop_status r = tc_up_only(&c->plan, a, c->tiles, c->status, st, &n);
+        c->launches += n;
+        return r;
+    }
+    ScalarGemmArgs g{};
+    g.A[0] = g.A[1] = static_cast<const bf16*>(Xp);
+    g.B[0] = static_cast<const bf16*>(W_gate); g.B[1] = static_cast<const bf16*>(W_up);
+    g.sAm = s.d; g.sAk = 1; g.sBk = s.f; g.sBn = 1; g.sBe = (long)s.d * s.f;
+    g.offsets = offsets; g.ragged_k = 0; g.N = s.f; g.Kfix = s.d; g.npairs = 2; g.dual_acc = 1; g.epi = EPI_SWIGLU;
+    g.ep.out0 = static_cast<bf16*>(H); g.ep.out1 = static_cast<bf16*>(G_save); g.ep.out2 = static_cast<bf16*>(U_save);
+    g.ep.ldo = s.f; g.ep.M_total = M;
+    return launch_scalar(c, "scalar_up_swiglu", g, st);
+}
+}  // namespace
+
 mop_status mop_moe_expert_ffn_fwd(mop_ctx* c, const void* Xp, const int32_t* offsets, const int32_t* row_src,
                                   const float* topk_gate, const void* W_gate, const void* W_up, const void* W_down,
                                   void* G_save, void* U_save, void* H, void* Yp, void* stream) {
@@ -437,7 +476,12 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
                                   float* dW_down, float* dgate, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
     if (!c->s.with_backward) return MOP_ERR_UNSUPPORTED;
-    REQ_PTR_T(dY); REQ_PTR_T(Xp); REQ_PTR_T(G_save); REQ_PTR_T(U_save); REQ_PTR_T(H); REQ_PTR(offsets);
+    // Recompute mode (activation checkpointing): with G_save, U_save and H all NULL the up-projection is
+    // run again from Xp into the context's own buffers (the same kernel as the forward: same bits).
+    const bool recompute = c->s.T > 0 && !G_save && !U_save && !H;
+    if (recompute && c->s.with_backward != 2) return MOP_ERR_UNSUPPORTED;
+    REQ_PTR_T(dY); REQ_PTR_T(Xp); REQ_PTR(offsets);
+    if (!recompute) { REQ_PTR_T(G_save); REQ_PTR_T(U_save); REQ_PTR_T(H); }
     REQ_PTR_T(perm_row); REQ_PTR_T(row_src); REQ_PTR_T(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up); REQ_PTR(W_down);
     REQ_PTR_T(dX); REQ_PTR(dW_gate); REQ_PTR(dW_up); REQ_PTR(dW_down); REQ_PTR_T(dgate);
     const mop_moe_shape& s = c->s;
@@ -446,6 +490,10 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int M = s.T * s.k;
     mop_status r;
+    if (recompute && s.T > 0) {
+        if ((r = up_projection(c, Xp, offsets, W_gate, W_up, c->rG, c->rU, c->rH, st)) != MOP_OK) return r;
+        G_save = c->rG; U_save = c->rU; H = c->rH;
+    }
     if (s.T > 0) {
         // dYp[p,:] = dY[t,:]  (unscaled; the gate enters through dH and gate*H)
         const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);

@@ -237,3 +237,28 @@ def test_router_backward_matches_oracle(w):
     got = dX.float().cpu().numpy()
     assert np.max(np.abs(got - want)) <= 2.0 ** -8 * np.maximum(1.0, np.abs(want)).max()
     assert rel_fro(got, want) < 4e-3
+
+
+def test_backward_with_recomputation_equals_backward_with_stash():
+    """Activation checkpointing: forward without the G, U stash, backward recomputes them from Xp."""
+    w = synth.small("c2_mid", T=700, d=256, E=10, k=3, f=192, backward=True, seed=40)
+    host, inp, _, ref = run(w)
+    ctx = binding.Context(w.T, w.d, w.E, w.k, w.f, w.score_fn, w.bias_mode, 2)
+    buf = binding.LayerBuffers(w)
+    binding.mop_moe_route(ctx, inp["x"], inp["W_r"], inp["bias"], buf.idx, buf.gate)
+    binding.mop_moe_permute(ctx, inp["x"], buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, buf.Xp)
+    binding.mop_moe_expert_ffn_fwd(ctx, buf.Xp, buf.offsets, buf.row_src, buf.gate, inp["W_gate"], inp["W_up"],
+                                   inp["W_down"], None, None, buf.H, buf.Yp)
+    binding.mop_moe_combine(ctx, buf.Yp, buf.perm_row, buf.Y)
+    binding.mop_moe_expert_ffn_bwd(ctx, inp["dY"], buf.Xp, None, None, None, buf.offsets, buf.perm_row, buf.row_src,
+                                   buf.gate, inp["W_gate"], inp["W_up"], inp["W_down"], buf.dX, buf.dW_gate, buf.dW_up,
+                                   buf.dW_down, buf.dgate)
+    binding.mop_poll(ctx)
+    for n in ("Y", "dX", "dgate", "dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(getattr(buf, n), getattr(ref, n)), n
+    plain = binding.context_for(w)                      # a context without the recompute buffers refuses
+    with pytest.raises(binding.MopError) as e:
+        binding.mop_moe_expert_ffn_bwd(plain, inp["dY"], buf.Xp, None, None, None, buf.offsets, buf.perm_row,
+                                       buf.row_src, buf.gate, inp["W_gate"], inp["W_up"], inp["W_down"], buf.dX,
+                                       buf.dW_gate, buf.dW_up, buf.dW_down, buf.dgate)
+    assert e.value.code == 6
