@@ -262,3 +262,21 @@ def test_backward_with_recomputation_equals_backward_with_stash():
                                        buf.row_src, buf.gate, inp["W_gate"], inp["W_up"], inp["W_down"], buf.dX,
                                        buf.dW_gate, buf.dW_up, buf.dW_down, buf.dgate)
     assert e.value.code == 6
+
+
+def test_random_small_shapes_match_oracle():
+    """Seeded random shapes: E not a multiple of 32, k from 1 to E, d and f multiples of 8 (scalar
+    kernels) or of 64 (tensor-core kernels), tokens that leave experts empty."""
+    rng = np.random.default_rng(1234)
+    for i in range(10):
+        E = int(rng.integers(1, 70))
+        k = int(rng.integers(1, min(E, 8) + 1))
+        if i % 2:
+            d, f = int(rng.integers(1, 5)) * 64, int(rng.integers(1, 5)) * 64
+        else:
+            d, f = int(rng.integers(2, 20)) * 8, int(rng.integers(2, 20)) * 8
+        T = int(rng.integers(1, 400))
+        mode = [(0, 0), (1, 1), (1, 2), (0, 2), (1, 0)][i % 5]
+        w = synth.small("c1_tiny", T=T, d=d, E=E, k=k, f=f, score_fn=mode[0], bias_mode=mode[1], bias_std=0.05,
+                        backward=True, seed=100 + i)
+        check_layer(w, binding.GEMM_AUTO)
