@@ -83,6 +83,12 @@ const char* mop_status_string(mop_status s);
  * exhausted wait since the last poll (then clears the word), MOP_ERR_CUDA on a CUDA error. */
 mop_status mop_poll(mop_ctx* ctx, void* stream);
 
+/* Self-test of the failure path: launches one thread that waits on a barrier nothing completes, with
+ * a limit of `limit_cycles` SM cycles (<= 4e9), synchronises, and returns MOP_OK if the wait gave up
+ * and the kernel ended normally.  The kernel records its code in the status word, so the next
+ * mop_poll on this context returns MOP_ERR_TIMEOUT (and clears it).  Nothing faults or traps. */
+mop_status mop_selftest_wait_timeout(mop_ctx* ctx, int64_t limit_cycles, void* stream);
+
 /* Number of kernels launched through this context since it was created. */
 int64_t mop_launch_count(const mop_ctx* ctx);
 

@@ -51,6 +51,7 @@ def lib() -> ctypes.CDLL:
         L.mop_destroy.restype = None
         L.mop_poll.argtypes = [_P, _P]
         L.mop_launch_count.argtypes = [_P]
+        L.mop_selftest_wait_timeout.argtypes = [_P, ctypes.c_int64, _P]
         L.mop_launch_count.restype = ctypes.c_int64
         L.mop_moe_route.argtypes = [_P] * 8
         L.mop_moe_permute.argtypes = [_P] * 9
@@ -121,6 +122,10 @@ class Context:
 
 def mop_poll(ctx, stream=None):
     _check("mop_poll", lib().mop_poll(ctx.handle, _stream(stream)))
+
+
+def mop_selftest_wait_timeout(ctx, limit_cycles=20_000_000, stream=None):
+    _check("mop_selftest_wait_timeout", lib().mop_selftest_wait_timeout(ctx.handle, limit_cycles, _stream(stream)))
 
 
 def mop_moe_route(ctx, x, W_r, bias, topk_idx, topk_gate, logits=None, stream=None):

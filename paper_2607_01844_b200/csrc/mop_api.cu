@@ -311,6 +311,21 @@ void mop_destroy(mop_ctx* c) {
 
 int64_t mop_launch_count(const mop_ctx* c) { return c ? c->launches : 0; }
 
+mop_status mop_selftest_wait_timeout(mop_ctx* c, int64_t limit_cycles, void* stream) {
+    if (!c || limit_cycles < 1 || limit_cycles > 4000000000ll) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* gave_up = c->status + 8;                    // a spare word of the status block
+    CUDA_OK(cudaMemsetAsync(gave_up, 0, 4, st));
+    tc_wait_selftest_kernel<<<1, 32, 0, st>>>(c->status, limit_cycles, gave_up);
+    if (after_launch(c) != MOP_OK) return MOP_ERR_CUDA;
+    int32_t flag = 0;
+    CUDA_OK(cudaMemcpyAsync(&flag, gave_up, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    return flag == 1 ? MOP_OK : MOP_ERR_CUDA;            // the wait must have given up, not completed
+}
+
 mop_status mop_poll(mop_ctx* c, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);

@@ -280,3 +280,23 @@ def test_random_small_shapes_match_oracle():
         w = synth.small("c1_tiny", T=T, d=d, E=E, k=k, f=f, score_fn=mode[0], bias_mode=mode[1], bias_std=0.05,
                         backward=True, seed=100 + i)
         check_layer(w, binding.GEMM_AUTO)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """Failure path without a fault: a device-side wait on a barrier that nothing completes gives up
+    after its limit, records a code, the kernel returns; mop_poll reports MOP_ERR_TIMEOUT once, and
+    the same context then runs the layer correctly."""
+    w = synth.small("c1_tiny", backward=True)
+    host = synth.make_inputs(w, "cpu")
+    inp = to_dev(host)
+    ctx = binding.context_for(w)
+    buf = binding.LayerBuffers(w)
+    binding.mop_selftest_wait_timeout(ctx, 20_000_000)          # about 10 ms of SM cycles
+    with pytest.raises(binding.MopError) as e:
+        binding.mop_poll(ctx)
+    assert e.value.code == 7
+    binding.mop_poll(ctx)                                        # the word was cleared
+    binding.forward(ctx, inp, buf)
+    binding.backward(ctx, inp, buf)
+    binding.mop_poll(ctx)
+    check_integers(w, host, buf)
