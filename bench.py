@@ -38,8 +38,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
 # (kernel, workload).  Filled from the summaries under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES: dict = {
-    # profiles/gemm_wgrad_gate_up_c5shape_E16.md: (63.8 MB read + 1819.5 MB written) at E = 16, x 384/16
-    ("gemm_wgrad_gate_up", "c5_train"): 24 * (63.774208e6 + 1.819528e9),
+    # profiles/gemm_wgrad_gate_up_c5shape_E16.md: (66.0 MB read + 1820.9 MB written) at E = 16, x 384/16
+    ("gemm_wgrad_gate_up", "c5_train"): 24 * (66.024448e6 + 1.820895e9),
 }
 
 
