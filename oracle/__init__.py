@@ -276,3 +276,17 @@ def route_bwd(x_bits, W_r, bias, k, score_fn, bias_mode, idx, dgate):
     np.put_along_axis(dz, idx, dzs, 1)
     dbias = dz.sum(0) if bias_mode == BIAS_PRE_LOGIT else np.zeros(E)
     return dz, x.T @ dz, dz @ W.T, dbias
+
+
+# ----------------------------------------------------------------------------- vocabulary projection
+def vocab_loss(x_bits, W_bits, targets):
+    """Per-token log-likelihood of the vocabulary projection (plain numpy, fp64):
+        Y = X W_voc  [N,V],   loss[n] = Y[n, t_n] - log sum_v exp(Y[n, v]).
+    x_bits [N,H], W_bits [H,V] bf16 bit patterns, targets [N] int.  Returns (loss [N], lse [N])."""
+    X = bf16_bits_to_f64(x_bits)
+    W = bf16_bits_to_f64(W_bits)
+    t = np.asarray(targets, np.int64)
+    Y = X @ W
+    m = Y.max(1)
+    lse = m + np.log(np.exp(Y - m[:, None]).sum(1))
+    return Y[np.arange(Y.shape[0]), t] - lse, lse

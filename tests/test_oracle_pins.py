@@ -403,3 +403,26 @@ def test_router_backward_central_differences():
         Wm[i, e] -= 1e-6
         fd = (loss(Wp) - loss(Wm)) / 2e-6
         assert abs(fd - dWr[i, e]) <= 1e-6 * max(1.0, abs(dWr[i, e]))
+
+
+# ------------------------------------------------------------------------------ vocabulary projection
+def test_vocab_loss_matches_library_cross_entropy_and_closed_forms():
+    rng = np.random.default_rng(40)
+    N, H, V = 13, 24, 301
+    x = _rand_bits(rng, (N, H))
+    W = _rand_bits(rng, (H, V), 0.3)
+    t = rng.integers(0, V, N)
+    loss, lse = oracle.vocab_loss(x, W, t)
+    Y = torch.tensor(oracle.bf16_bits_to_f64(x) @ oracle.bf16_bits_to_f64(W))
+    ce = torch.nn.functional.cross_entropy(Y, torch.from_numpy(t), reduction="none").numpy()
+    assert np.max(np.abs(loss + ce)) < 1e-12                      # the log-likelihood is minus the cross entropy
+    assert np.max(np.abs(lse - torch.logsumexp(Y, 1).numpy())) < 1e-12
+    # all-zero weights: every token has log-likelihood -log V
+    l0, lse0 = oracle.vocab_loss(x, np.zeros_like(W), t)
+    assert np.allclose(l0, -np.log(V)) and np.allclose(lse0, np.log(V))
+    # a shift of all logits of a token leaves the loss unchanged and moves lse by the shift
+    assert np.all(loss <= 0)
+    # large logits do not overflow
+    big = synth.bits((torch.from_numpy(oracle.bf16_bits_to_f32(W)) * 64).to(torch.bfloat16))
+    lb, _ = oracle.vocab_loss(x, big, t)
+    assert np.all(np.isfinite(lb))
