@@ -195,6 +195,19 @@ mop_status mop_profile_enable(mop_ctx* ctx, int on);
 int32_t mop_profile_read(mop_ctx* ctx, void* stream, int32_t max_names, const char** names, float* total_ms,
                          int32_t* calls);
 
+/* Vocabulary projection with an online loss (Eq. 5 of the paper): with X [N,H] and W_voc [H,V],
+ *   Y = X W_voc,   loss[n] = Y[n, t_n] - log sum_v exp(Y[n, v])      (the token's log-likelihood)
+ * computed tile by tile on the tensor cores (bf16 operands, fp32 accumulation) with a running
+ * maximum and sum per row, so that the N x V logits are never stored: the only intermediate is one
+ * (max, sum) pair per row and 256-column block.  One-GPU counterpart of Section 3.4's projection;
+ * forward only.  H and V must be multiples of 64.
+ * X [N,H] bf16; W_voc [H,V] bf16; targets [N] i32 in [0,V); loss [N] f32 out; lse_opt [N] f32 out or
+ * NULL; workspace: device memory of mop_vocab_workspace_bytes(N, H, V) bytes, 256-byte aligned,
+ * owned by the caller (nothing is allocated here).  `device` is the CUDA ordinal. */
+size_t mop_vocab_workspace_bytes(int32_t N, int32_t H, int32_t V);
+mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const void* X, const void* W_voc,
+                              const int32_t* targets, float* loss, float* lse_opt, void* workspace, void* stream);
+
 /* The same permutation as mop_moe_permute for callers that may not allocate device memory (the
  * paper has no counterpart; this is a property of the library, not of the method).  A process
  * that gave all of HBM to its own arena, or a loop that cannot take the device-wide

@@ -62,6 +62,9 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_route_bwd.argtypes = [_P] * 14
         L.mop_moe_train_step_host.argtypes = [_P] * 15
         L.mop_moe_permute_static.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 4 + [_P] * 8
+        L.mop_vocab_workspace_bytes.argtypes = [ctypes.c_int32] * 3
+        L.mop_vocab_workspace_bytes.restype = ctypes.c_size_t
+        L.mop_vocab_loss_fwd.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 3 + [_P] * 7
         L.mop_profile_enable.argtypes = [_P, ctypes.c_int]
         L.mop_profile_read.argtypes = [_P, _P, ctypes.c_int32, ctypes.POINTER(ctypes.c_char_p),
                                        ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
@@ -189,6 +192,22 @@ def mop_moe_permute_static(device, T, d, E, k, x, topk_idx, counts, offsets, per
     _check("mop_moe_permute_static",
            lib().mop_moe_permute_static(device, T, d, E, k, _ptr(x), _ptr(topk_idx), _ptr(counts), _ptr(offsets),
                                         _ptr(perm_row), _ptr(row_src), _ptr(Xp), _stream(stream)))
+
+
+def mop_vocab_workspace_bytes(N, H, V):
+    return lib().mop_vocab_workspace_bytes(N, H, V)
+
+
+def mop_vocab_loss_fwd(device, X, W_voc, targets, loss, lse=None, workspace=None, stream=None):
+    """loss[n] = (X W_voc)[n, t_n] - logsumexp_v (X W_voc)[n, v]; the logits are never stored."""
+    N, H = X.shape
+    V = W_voc.shape[1]
+    if workspace is None:
+        workspace = torch.empty(max(256, mop_vocab_workspace_bytes(N, H, V)), dtype=torch.uint8, device=X.device)
+    _check("mop_vocab_loss_fwd",
+           lib().mop_vocab_loss_fwd(device, N, H, V, _ptr(X), _ptr(W_voc), _ptr(targets), _ptr(loss), _ptr(lse),
+                                    _ptr(workspace), _stream(stream)))
+    return workspace
 
 
 def mop_profile_enable(ctx, on=True):

@@ -8,6 +8,7 @@
 //   B4   dXp   = dG W_gate[e]^T + dU W_up[e]^T    (two K phases)  -> bf16             ragged M
 //   WD   dW_down[e] = (gate H)_e^T dYp_e          fp32 store                          ragged K
 //   WGU  [dW_gate|dW_up][e] = Xp_e^T [dG|dU]_e    fp32 store                          ragged K
+//   VL   Y = X W_voc (never stored)               online log-sum-exp partials         dense M
 // CTA tile 128 x 256 (one tcgen05.mma.cta_group::1 of M=128, N=256, K=16 per 32 bytes of K),
 // K step 64 per pipeline stage, 4 stages, two 256-column accumulators in TMEM so that the
 // epilogue of tile i overlaps the main loop of tile i+1.
@@ -23,7 +24,7 @@
 
 namespace mop {
 
-enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5 };
+enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5, TC_VL = 6 };
 
 constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // 16 KiB
@@ -60,6 +61,9 @@ struct TcArgs {
     int tiles_m_fixed;       // ragged K: m-tiles per expert
     int kblocks;             // ragged M: K / 64 (rounded up) per phase
     int Mfix, N;             // ragged K: output rows per expert; N = columns per output tensor
+    int m_fastest;           // tile order: 1 = consecutive tiles walk the row tiles of one column block
+    const int32_t* targets;  // VL: target column per row
+    float* ylab;             // VL: logit of the target column per row
     int32_t* status;
     EpiArgs ep;
     float* outf1;            // WGU: second output tensor
@@ -274,9 +278,12 @@ __device__ __forceinline__ TileInfo decode_tile(const TcArgs& a, int t) {
         ti.rows = __ldg(a.offsets + ti.e + 1) - ti.row0;
         ti.skip = ti.rows <= 0;
     } else {
-        const int4 m = __ldg(a.mtiles + t / a.tiles_n);
+        int mt, nt;
+        if (a.m_fastest) { const int nm = __ldg(a.n_mtiles); nt = t / nm; mt = t - nt * nm; }
+        else { mt = t / a.tiles_n; nt = t - mt * a.tiles_n; }
+        const int4 m = __ldg(a.mtiles + mt);
         ti.e = m.x; ti.row0 = m.y; ti.rows = m.z; ti.m0 = 0;
-        ti.nt = t % a.tiles_n;
+        ti.nt = nt;
         ti.skip = false;
     }
     return ti;
@@ -345,6 +352,35 @@ __device__ __forceinline__ void tc_epilogue_rows(const TcArgs& args, uint32_t ta
             }
         }
         if (KIND == TC_B2 && row_ok) args.ep.part[(size_t)nt * args.ep.M_total + grow] = dot;
+    } else if constexpr (KIND == TC_VL) {
+        // Online log-sum-exp over this tile's 256 logits of the row (fp32 accumulators, never stored):
+        // running maximum m and s = sum exp(y - m); the target's logit is picked up where it falls.
+        float m = -INFINITY, ssum = 0.0f;
+        const int tgt = row_ok ? args.targets[grow] - n0 : -1;
+#pragma unroll 1
+        for (int c = 0; c < TC_BN; c += 32) {
+            tmem_ld32(taddr + c, acc);
+            if (row_ok && n0 + c < args.N) {
+                float cm = acc[0];
+#pragma unroll
+                for (int q = 1; q < 32; ++q) cm = fmaxf(cm, acc[q]);
+                const float nm = fmaxf(m, cm);
+                float part = 0.0f;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) part += __expf(acc[q] - nm);
+                ssum = ssum * __expf(m - nm) + part;
+                m = nm;
+                if (tgt >= c && tgt < c + 32) {
+                    float y = 0.0f;
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) y = (tgt - c == q) ? acc[q] : y;
+                    args.ylab[grow] = y;
+                }
+            }
+        }
+        if (row_ok) {
+            reinterpret_cast<float2*>(args.ep.part)[(size_t)nt * args.ep.M_total + grow] = make_float2(m, ssum);
+        }
     } else if constexpr (KIND == TC_B4) {
 #pragma unroll 1
         for (int c = 0; c < TC_BN; c += 32) {
@@ -617,6 +653,24 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
     }
 }
 
+// Merge of the per-tile (max, sum) pairs of a row: lse = M + log sum_i s_i exp(m_i - M); the
+// log-likelihood is the target's logit minus lse.  Fixed order: reproducible.
+__global__ void vocab_lse_merge_kernel(const float2* __restrict__ part, const float* __restrict__ ylab,
+                                       float* __restrict__ loss, float* __restrict__ lse, int N, int ntiles) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    float M = -INFINITY;
+    for (int i = 0; i < ntiles; ++i) M = fmaxf(M, part[(size_t)i * N + n].x);
+    float S = 0.0f;
+    for (int i = 0; i < ntiles; ++i) {
+        const float2 p = part[(size_t)i * N + n];
+        S += p.y * expf(p.x - M);
+    }
+    const float l = M + logf(S);
+    if (lse) lse[n] = l;
+    loss[n] = ylab[n] - l;
+}
+
 // ------------------------------------------------------------------------------------------ host
 struct TcPlan {
     int sm_count;
@@ -671,6 +725,7 @@ inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count, 
     if ((r = tc_set_smem<TC_B4>()) != MOP_OK) return r;
     if ((r = tc_set_smem<TC_WD>()) != MOP_OK) return r;
     if ((r = tc_set_smem<TC_WGU>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_VL>()) != MOP_OK) return r;
     return MOP_OK;
 }
 

@@ -803,4 +803,84 @@ mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, i
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Vocabulary projection + online log-likelihood (no context: the caller owns the workspace)
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct VocabLayout { size_t off, tiles, status, ylab, part, total; };
+VocabLayout vocab_layout(int N, int V) {
+    VocabLayout L{};
+    size_t o = 0;
+    auto take = [&](size_t b) { size_t r = o; o += align_up(b); return r; };
+    L.off = take(16);
+    L.tiles = take(tc_tile_table_bytes(N, 1));
+    L.status = take(256);
+    L.ylab = take((size_t)N * 4);
+    L.part = take((size_t)ceil_div(V, 256) * N * 8);
+    L.total = o;
+    return L;
+}
+std::mutex g_vocab_mutex;
+TcPlan g_vocab_plan[kMaxDevices];
+Profiler g_vocab_prof;           // never enabled: the plan needs one
+bool g_vocab_ready[kMaxDevices];
+}  // namespace
+
+size_t mop_vocab_workspace_bytes(int32_t N, int32_t H, int32_t V) {
+    if (N < 0 || H < 64 || V < 64 || H % 64 || V % 64) return 0;
+    return vocab_layout(N, V).total;
+}
+
+mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const void* X, const void* W_voc,
+                              const int32_t* targets, float* loss, float* lse_opt, void* workspace, void* stream) {
+    if (N < 0 || H < 1 || V < 1) return MOP_ERR_INVALID_ARG;
+    if (H % 64 || V % 64) return MOP_ERR_UNSUPPORTED;
+    if ((long long)N * 2 >= (1ll << 31) || (long long)H * V >= (1ll << 40)) return MOP_ERR_SHAPE;
+    if (N == 0) return MOP_OK;
+    if (!X || !W_voc || !targets || !loss || !workspace) return MOP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(W_voc) || !aligned16(targets) || !aligned16(loss) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255u) || (lse_opt && !aligned16(lse_opt)))
+        return MOP_ERR_ALIGN;
+    if (device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    TcPlan* p = &g_vocab_plan[device];
+    {
+        std::lock_guard<std::mutex> lock(g_vocab_mutex);
+        if (!g_vocab_ready[device]) {
+            cudaDeviceProp prop;
+            if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MOP_ERR_CUDA;
+            if (prop.major != 10) return MOP_ERR_UNSUPPORTED;
+            mop_moe_shape dummy{};
+            mop_status r = tc_plan_init(p, dummy, prop.multiProcessorCount, &g_vocab_prof);
+            if (r != MOP_OK) return r;
+            g_vocab_ready[device] = true;
+        }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const VocabLayout L = vocab_layout(N, V);
+    char* w = static_cast<char*>(workspace);
+    int32_t* off = reinterpret_cast<int32_t*>(w + L.off);
+    int32_t* tiles = reinterpret_cast<int32_t*>(w + L.tiles);
+    int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+    float* ylab = reinterpret_cast<float*>(w + L.ylab);
+    float* part = reinterpret_cast<float*>(w + L.part);
+    const int32_t host_off[2] = {0, N};
+    CUDA_OK(cudaMemcpyAsync(off, host_off, sizeof(host_off), cudaMemcpyHostToDevice, st));
+    CUDA_OK(cudaMemsetAsync(status, 0, 4, st));
+    tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
+    CUtensorMap mX, mW;
+    if (!tc_map_2d(p, &mX, X, N, H, 128) || !tc_map_chunked_3d(p, &mW, W_voc, 1, H, V, 4)) return MOP_ERR_CUDA;
+    TcArgs g{};
+    g.offsets = off; g.n_mtiles = tiles; g.mtiles = reinterpret_cast<const int4*>(tiles + 64);
+    g.E = 1; g.status = status;
+    g.tiles_n = ceil_div(V, 256); g.kblocks = ceil_div(H, TC_BK); g.N = V; g.m_fastest = 1;
+    g.targets = targets; g.ylab = ylab; g.ep.part = part; g.ep.M_total = N;
+    mop_status r = tc_launch<TC_VL>(p, "vocab_logits_lse", mX, mX, mW, mW, mX, mX, g, st);
+    if (r != MOP_OK) return r;
+    vocab_lse_merge_kernel<<<ceil_div(N, 256), 256, 0, st>>>(reinterpret_cast<const float2*>(part), ylab, loss,
+                                                            lse_opt, N, g.tiles_n);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
 }  // extern "C"
