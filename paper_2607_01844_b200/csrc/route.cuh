@@ -16,7 +16,8 @@ namespace mop {
 // (16 RT) tokens x (8 RE) experts; operands are staged through shared memory in slabs of 16 or 32
 // along i, double-buffered, the next slab prefetched into registers while the current one is
 // multiplied.  <8,8> needs 4 shared loads per 64 FMAs; smaller tiles trade that for more CTAs
-// when T*E is small.
+// when T*E is small.  Both slabs are laid out so that every shared access of a warp is free of
+// bank conflicts (interleaved expert columns, XOR-swizzled token columns).
 // ---------------------------------------------------------------------------------------------
 constexpr int SC_THREADS = 128;
 
@@ -33,7 +34,7 @@ __device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long
 }
 
 template <int RT, int RE, int SC_TK>
-__global__ void __launch_bounds__(SC_THREADS) route_score_kernel(const bf16* __restrict__ x,
+__global__ void __launch_bounds__(SC_THREADS, 4) route_score_kernel(const bf16* __restrict__ x,
                                                                  const float* __restrict__ W_r,
                                                                  float* __restrict__ z, int T, int d, int E) {
     constexpr int TT = 16 * RT, TE = 8 * RE;          // CTA tile
@@ -45,7 +46,14 @@ __global__ void __launch_bounds__(SC_THREADS) route_score_kernel(const bf16* __r
     __shared__ __align__(16) float ws[2][SC_TK][LDW];
     const int t0 = blockIdx.x * TT, e0 = blockIdx.y * TE;
     const int tid = threadIdx.x;
-    const int tt = (tid / 8) * RT, te = (tid % 8) * RE;
+    // Expert columns of a thread: groups of 4 at te + 32 b, so that the 8 threads that differ in
+    // tid % 8 read 32 consecutive floats (one conflict-free wavefront) per group.
+    const int tt = (tid / 8) * RT, te = (tid % 8) * 4;
+    constexpr int EG = (RE > 4) ? 32 : 4;             // column pitch between a thread's groups of 4
+    // Token columns of the x slab are XOR-swizzled by the 8-row chunk of i they belong to: the
+    // threads of a warp that stash different chunks of the same tokens then hit different banks.
+    constexpr int CH = SC_TK / 8, SWZ = 32 / CH;
+    static_assert(TT >= 32 && (SWZ % 4) == 0, "swizzle keeps float4 groups intact and stays inside the tile");
     const bool w_vec = (E % 4 == 0);
 
     unsigned long long acc[RT / 2][RE];   // acc[a][b] = chains of tokens (2a, 2a+1) for expert b
@@ -90,8 +98,8 @@ __global__ void __launch_bounds__(SC_THREADS) route_score_kernel(const bf16* __r
             const uint32_t w4[4] = {xr[v].x, xr[v].y, xr[v].z, xr[v].w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                xs[buf][ii + 2 * q][tok] = bf16_lo(w4[q]);
-                xs[buf][ii + 2 * q + 1][tok] = bf16_hi(w4[q]);
+                xs[buf][ii + 2 * q][tok ^ ((ii / 8) * SWZ)] = bf16_lo(w4[q]);
+                xs[buf][ii + 2 * q + 1][tok ^ ((ii / 8) * SWZ)] = bf16_hi(w4[q]);
             }
         }
 #pragma unroll
@@ -114,17 +122,17 @@ __global__ void __launch_bounds__(SC_THREADS) route_score_kernel(const bf16* __r
             unsigned long long xp[RT / 2], wp[RE];
 #pragma unroll
             for (int a = 0; a < RT / 4; ++a) {
-                const float4 v = *reinterpret_cast<const float4*>(&xs[buf][kk][tt + 4 * a]);
+                const float4 v = *reinterpret_cast<const float4*>(&xs[buf][kk][(tt + 4 * a) ^ ((kk / 8) * SWZ)]);
                 xp[2 * a] = pack_f32x2(v.x, v.y);
                 xp[2 * a + 1] = pack_f32x2(v.z, v.w);
             }
             if constexpr (RT % 4 == 2) {
-                const float2 v = *reinterpret_cast<const float2*>(&xs[buf][kk][tt + RT - 2]);
+                const float2 v = *reinterpret_cast<const float2*>(&xs[buf][kk][(tt + RT - 2) ^ ((kk / 8) * SWZ)]);
                 xp[RT / 2 - 1] = pack_f32x2(v.x, v.y);
             }
 #pragma unroll
             for (int b = 0; b < RE / 4; ++b) {
-                const float4 v = *reinterpret_cast<const float4*>(&ws[buf][kk][te + 4 * b]);
+                const float4 v = *reinterpret_cast<const float4*>(&ws[buf][kk][te + EG * b]);
                 wp[4 * b] = pack_f32x2(v.x, v.x);
                 wp[4 * b + 1] = pack_f32x2(v.y, v.y);
                 wp[4 * b + 2] = pack_f32x2(v.z, v.z);
@@ -148,18 +156,19 @@ __global__ void __launch_bounds__(SC_THREADS) route_score_kernel(const bf16* __r
         for (int h = 0; h < 2; ++h) {
             const int t = t0 + tt + 2 * a + h;
             if (t >= T) continue;
-            float* dst = z + (size_t)t * E + e0 + te;
 #pragma unroll
             for (int b = 0; b < RE; b += 4) {
                 const float v0 = h ? hi[b] : lo[b], v1 = h ? hi[b + 1] : lo[b + 1];
                 const float v2 = h ? hi[b + 2] : lo[b + 2], v3 = h ? hi[b + 3] : lo[b + 3];
-                if (w_vec && e0 + te + b + 3 < E) {
-                    *reinterpret_cast<float4*>(dst + b) = make_float4(v0, v1, v2, v3);
+                const int e = e0 + te + EG * (b / 4);
+                float* dst = z + (size_t)t * E + e;
+                if (w_vec && e + 3 < E) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(v0, v1, v2, v3);
                 } else {
-                    if (e0 + te + b < E) dst[b] = v0;
-                    if (e0 + te + b + 1 < E) dst[b + 1] = v1;
-                    if (e0 + te + b + 2 < E) dst[b + 2] = v2;
-                    if (e0 + te + b + 3 < E) dst[b + 3] = v3;
+                    if (e < E) dst[0] = v0;
+                    if (e + 1 < E) dst[1] = v1;
+                    if (e + 2 < E) dst[2] = v2;
+                    if (e + 3 < E) dst[3] = v3;
                 }
             }
         }
