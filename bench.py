@@ -70,6 +70,7 @@ def kernel_work(w, counts):
         "dy_scatter_rows": (0, T * d * 2 + M * d * 2 + M * 4),
         "combine_rows": (0, M * d * 2 + T * d * 2 + M * 4),
         "gemm_up_swiglu": (4 * mdf, live * 2 * d * f * 2 + M * d * 2 + stash * M * f * 2),
+        "gemm_up_swiglu_gather": (4 * mdf, live * 2 * d * f * 2 + T * d * 2 + M * f * 2),
         "gemm_down_gate": (2 * mdf, live * d * f * 2 + M * f * 2 + M * d * 2),
         "gemm_dgrad_down_dswiglu": (2 * mdf, live * d * f * 2 + M * d * 2 + 6 * M * f * 2),
         "gemm_dgrad_gate_up": (4 * mdf, live * 2 * d * f * 2 + 2 * M * f * 2 + M * d * 2),
@@ -257,6 +258,8 @@ def main():
     ap.add_argument("--gemm-path", type=int, default=0, help="mop_gemm_path (0 = library default)")
     ap.add_argument("--with-router-bwd", action="store_true",
                     help="also run the router backward (dgate -> dW_r, dX) in every step of a fwd+bwd workload")
+    ap.add_argument("--gather", action="store_true",
+                    help="forward-only workloads: up-projection gathers its rows from x (no permuted copy)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -302,7 +305,7 @@ def main():
                                            inp["W_down"], buf.G, buf.U, buf.H, buf.Yp, stream)
             binding.mop_moe_combine(ctx, buf.Yp, buf.perm_row, buf.Y, stream)
         else:
-            binding.forward(ctx, inp, buf, stream)
+            binding.forward(ctx, inp, buf, stream, gather=args.gather and not w.backward)
         if w.backward:
             binding.backward(ctx, inp, buf, stream)
         if rbwd:

@@ -108,7 +108,8 @@ mop_status mop_moe_route(mop_ctx* ctx, const void* x, const float* W_r, const fl
  *   perm_row[a] = offsets[idx[a]] + (number of a' < a with the same expert)     (stable)
  *   row_src     = inverse of perm_row;   Xp[p,:] = x[row_src[p] / k, :]
  * x [T,d] bf16; topk_idx [T,k]; counts [E]; offsets [E+1]; perm_row, row_src [T*k] i32 out;
- * Xp [T*k,d] bf16 out.  Indices outside [0,E) are a caller error (rows are dropped). */
+ * Xp [T*k,d] bf16 out, or NULL: only the tables are built (x is then not read), for
+ * mop_moe_expert_ffn_fwd_gather.  Indices outside [0,E) are a caller error (rows are dropped). */
 mop_status mop_moe_permute(mop_ctx* ctx, const void* x, const int32_t* topk_idx, int32_t* counts, int32_t* offsets,
                            int32_t* perm_row, int32_t* row_src, void* Xp, void* stream);
 
@@ -123,6 +124,19 @@ mop_status mop_moe_permute(mop_ctx* ctx, const void* x, const int32_t* topk_idx,
 mop_status mop_moe_expert_ffn_fwd(mop_ctx* ctx, const void* Xp, const int32_t* offsets, const int32_t* row_src,
                                   const float* topk_gate, const void* W_gate, const void* W_up, const void* W_down,
                                   void* G_save, void* U_save, void* H, void* Yp, void* stream);
+
+/* The same forward without the expert-contiguous copy of the inputs: the up-projection fetches
+ * row p of expert e straight from x[row_src[p] / k, :] while it stages its operand tiles, so Xp
+ * is never written or read (the N k H term of Eq. 4 drops out of the activation peak; the
+ * single-GPU counterpart of keeping only a fraction of the routed inputs resident, Section 3.3).
+ * Results are bit-identical to mop_moe_permute + mop_moe_expert_ffn_fwd.  No stash is written:
+ * this is the inference form.  Needs the tensor-core path (MOP_ERR_UNSUPPORTED otherwise).
+ * It trades time for memory: 4-row gather copies keep the TMA unit busier than 128-row boxes, and
+ * the up-projection takes about 2.4 times as long as in the permuting form.
+ * x [T,d] bf16; the other arguments as above. */
+mop_status mop_moe_expert_ffn_fwd_gather(mop_ctx* ctx, const void* x, const int32_t* offsets,
+                                         const int32_t* row_src, const float* topk_gate, const void* W_gate,
+                                         const void* W_up, const void* W_down, void* H, void* Yp, void* stream);
 
 /* Unpermute-combine: Y[t,:] = bf16( sum_j Yp[perm_row[t*k+j], :] ), fp32 sum, j ascending.
  * (The gate was applied by mop_moe_expert_ffn_fwd.)  Also used for dX from dXp.

@@ -56,6 +56,7 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_route.argtypes = [_P] * 8
         L.mop_moe_permute.argtypes = [_P] * 9
         L.mop_moe_expert_ffn_fwd.argtypes = [_P] * 13
+        L.mop_moe_expert_ffn_fwd_gather.argtypes = [_P] * 11
         L.mop_moe_combine.argtypes = [_P] * 5
         L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 19
         L.mop_moe_forward_host.argtypes = [_P] * 11
@@ -147,6 +148,13 @@ def mop_moe_expert_ffn_fwd(ctx, Xp, offsets, row_src, topk_gate, W_gate, W_up, W
            lib().mop_moe_expert_ffn_fwd(ctx.handle, _ptr(Xp), _ptr(offsets), _ptr(row_src), _ptr(topk_gate),
                                         _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(G_save), _ptr(U_save), _ptr(H),
                                         _ptr(Yp), _stream(stream)))
+
+
+def mop_moe_expert_ffn_fwd_gather(ctx, x, offsets, row_src, topk_gate, W_gate, W_up, W_down, H, Yp, stream=None):
+    _check("mop_moe_expert_ffn_fwd_gather",
+           lib().mop_moe_expert_ffn_fwd_gather(ctx.handle, _ptr(x), _ptr(offsets), _ptr(row_src), _ptr(topk_gate),
+                                               _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(H), _ptr(Yp),
+                                               _stream(stream)))
 
 
 def mop_moe_combine(ctx, Yp, perm_row, Y, stream=None):
@@ -256,9 +264,16 @@ class LayerBuffers:
             self.dW_down = torch.empty((E, f, d), **f32)
 
 
-def forward(ctx, inp, buf, stream=None):
+def forward(ctx, inp, buf, stream=None, gather=False):
     """route -> permute -> expert_ffn_fwd -> combine on device tensors (one pass of the forward path)."""
     mop_moe_route(ctx, inp["x"], inp["W_r"], inp["bias"], buf.idx, buf.gate, None, stream)
+    if gather:
+        # inference form: no expert-contiguous copy of x, no stash
+        mop_moe_permute(ctx, None, buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, None, stream)
+        mop_moe_expert_ffn_fwd_gather(ctx, inp["x"], buf.offsets, buf.row_src, buf.gate, inp["W_gate"], inp["W_up"],
+                                      inp["W_down"], buf.H, buf.Yp, stream)
+        mop_moe_combine(ctx, buf.Yp, buf.perm_row, buf.Y, stream)
+        return
     mop_moe_permute(ctx, inp["x"], buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, buf.Xp, stream)
     mop_moe_expert_ffn_fwd(ctx, buf.Xp, buf.offsets, buf.row_src, buf.gate, inp["W_gate"], inp["W_up"], inp["W_down"],
                            buf.G, buf.U, buf.H, buf.Yp, stream)

@@ -61,7 +61,8 @@ inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles,
     const uint64_t M = (uint64_t)s.T * s.k;
     mop_status r;
     // Tokens-on-N kernels: fwd_tn bit 0 = up-projection, bit 1 = down-projection (see tc_plan_policy)
-    const bool tn_f1 = p->fwd_tn & 1, tn_f2 = p->fwd_tn & 2;
+    const bool gather = a.x_gather != nullptr;
+    const bool tn_f1 = gather || (p->fwd_tn & 1), tn_f2 = p->fwd_tn & 2;
     if (tn_f1 || tn_f2) {
         if ((r = tn_build_tiles(p, a.offsets, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), st)) != MOP_OK) return r;
         ++*launches;
@@ -73,12 +74,15 @@ inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles,
     // N-major weights as chunked maps: one-CTA tiles take 2 chunks per tensor (gate | up) or 4 (down);
     // a pair CTA takes 2 chunks
     CUtensorMap mXp, mWg, mWu, mH, mWd, mWdp;
-    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, 128) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 2) ||
+    if ((!tn_f1 && !tc_map_2d(p, &mXp, a.Xp, M, s.d, 128)) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 2) ||
         !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 2) || !tc_map_2d(p, &mH, a.H, M, s.f, 128) ||
         !tc_map_chunked_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 4) ||
         !tc_map_chunked_3d(p, &mWdp, a.W_down, s.E, s.f, s.d, 2))
         return MOP_ERR_CUDA;
-    if (tn_f1) {
+    if (gather) {
+        if ((r = tn_up_swiglu_gather(p, a.x_gather, a, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), status, st)) != MOP_OK) return r;
+        ++*launches;
+    } else if (tn_f1) {
         if ((r = tn_up_swiglu(p, a, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), status, st)) != MOP_OK) return r;
         ++*launches;
     } else {   // F1: [G|U] = Xp [W_gate | W_up], SwiGLU epilogue

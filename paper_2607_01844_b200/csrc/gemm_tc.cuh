@@ -685,6 +685,7 @@ struct TcFwdArgs {
     const bf16* Xp; const int32_t* offsets; const int32_t* row_src; const float* gate;
     const bf16 *W_gate, *W_up, *W_down;
     bf16 *G_save, *U_save, *H, *Yp;
+    const bf16* x_gather;   // non-null: the up-projection gathers its rows from x [T, d] and Xp is unused
 };
 struct TcBwdArgs {
     const bf16 *dYp, *Xp, *G_save, *U_save, *H;

@@ -11,6 +11,12 @@
 //          l and l + 64); the epilogue exchanges U through shared memory, applies SwiGLU and
 //          writes H (+ G, U stash) back in token-major layout.
 //   TN_F2  O^T = W_down^T-tile * H^T, gate applied per token column, Yp written token-major.
+//   TN_F1G as TN_F1, but the token operand is gathered straight from the unpermuted x [T, d]: every
+//          lane of the producer warp owns four token rows of the tile and fetches them per K block
+//          with one TMA gather4 copy, so the expert-contiguous copy Xp never exists (the
+//          single-GPU form of keeping only a fraction of the routed inputs live, Section 3.3).
+//          The TMA unit retires these 4-row copies far more slowly than one 128-row box (about
+//          60 ns each on B200), so this form trades time for memory and is opt-in.
 //
 // The epilogue transposes 32 x 32 blocks through shared memory so that global stores are 64-byte
 // row segments.  Barrier protocol, bounded waits and teardown as in the pair kernel.
@@ -19,7 +25,7 @@
 
 namespace mop {
 
-enum : int { TN_F1 = 0, TN_F2 = 1 };
+enum : int { TN_F1 = 0, TN_F2 = 1, TN_F1G = 2 };
 
 constexpr int TN_STAGES = 5;
 constexpr int TN_A_BYTES = 128 * TC_BK * 2;          // 16 KiB: this CTA's 128 weight rows
@@ -36,6 +42,8 @@ struct TnArgs {
     int tiles_m;              // weight-row tiles per token tile (each 256 rows; F1: 128 columns of f)
     int kblocks;              // K / 64 rounded up
     int Mw;                   // weight rows in total (F1: f; F2: d)
+    const int32_t* row_src;   // F1G: assignment index t*k + j of every expert-contiguous row
+    int topk;                 // F1G: k (token of a row = row_src / k)
     int32_t* status;
     EpiArgs ep;
 };
@@ -61,6 +69,15 @@ __global__ void __launch_bounds__(1024) tn_build_ttiles_kernel(const int32_t* __
     const int sz = nt ? (((cnt + nt - 1) / nt + 15) & ~15) : 0;
     for (int i = 0; i < nt; ++i) tiles[first + i] = make_int4(e, off + i * sz, min(sz, cnt - i * sz), 0);
     if (e == 1023) *n_tiles = scan[1023];
+}
+
+// Four rows of a [rows, cols] bf16 tensor (map box {64, 1}) -> 4 x 128 bytes at dst, swizzled like a tile box.
+__device__ __forceinline__ void tma2_gather4(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int r0, int r1,
+                                             int r2, int r3) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes.cta_group::2 [%0], "
+        "[%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+        : "memory");
 }
 
 __device__ __forceinline__ void bar_pair_sync(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
@@ -108,7 +125,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB);
-        if (KIND == TN_F1) tma_prefetch_desc(&tmA1);
+        if (KIND != TN_F2) tma_prefetch_desc(&tmA1);
     }
     if (warp == 1) tmem2_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
@@ -128,7 +145,43 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         return ti;
     };
 
-    if (warp == 0) {
+    if (warp == 0 && KIND == TN_F1G) {
+        // ============================================ TMA producer with row gather (both CTAs, whole warp)
+        int stage = 0; uint32_t phase = 0; bool alive = true;
+        Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
+        for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
+            const Tile ti = nxt;
+            if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
+            const int half = ti.nmma >> 1;                             // token rows per CTA (multiple of 8)
+            const int ngroups = half >> 2;                             // gather4 copies per K block (<= 32)
+            const int brow0 = ti.row0 + (int)rank * half;
+            const int last = ti.row0 + ti.rows - 1;                    // padding rows repeat the last valid one
+            int tok[4] = {0, 0, 0, 0};
+            if (lane < ngroups) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) tok[j] = __ldg(args.row_src + min(brow0 + 4 * lane + j, last)) / args.topk;
+            }
+            const uint32_t tx = 2u * (TN_A_BYTES + (uint32_t)half * 128u);
+            for (int kb = 0; kb < args.kblocks; ++kb) {
+                if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY, lane)) {
+                    alive = false; break;
+                }
+                const uint32_t fb = full_bar(stage) & T2_PEER_MASK;
+                const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
+                const uint32_t sB = sA + TN_A_BYTES;
+                const int k0 = kb * TC_BK;
+                if (lane == 0) {
+                    if (leader) mbar_expect_tx(full_bar(stage), tx);
+                    const int f0 = ti.mt * 128 + 64 * (int)rank;
+                    tma2_load_4d(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e);
+                    tma2_load_4d(sA + TC_CHUNK_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e);
+                }
+                if (lane < ngroups) tma2_gather4(sB + lane * 512, &tmB, fb, k0, tok[0], tok[1], tok[2], tok[3]);
+                __syncwarp();
+                if (++stage == S) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 0) {
         // ===================================================================== TMA producer (both CTAs)
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool alive = true;
@@ -149,7 +202,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
                     const uint32_t sB = sA + TN_A_BYTES;
                     const int k0 = kb * TC_BK;
-                    if constexpr (KIND == TN_F1) {
+                    if constexpr (KIND != TN_F2) {
                         // 64 gate columns, then the 64 matching up columns (N-major weights [E, d, f])
                         const int f0 = ti.mt * 128 + 64 * (int)rank;
                         tma2_load_4d(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e);
@@ -220,7 +273,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256;
             float v[32];
 
-            if constexpr (KIND == TN_F1) {
+            if constexpr (KIND != TN_F2) {
                 // lanes 0..63 of the CTA hold gate rows, lanes 64..127 the matching up rows
                 const bool is_up = quarter >= 2;
                 const int fcol = ti.mt * 128 + 64 * (int)rank + 32 * (quarter & 1);   // first f of this warp
@@ -313,6 +366,8 @@ inline mop_status tn_init() {
     if (cudaFuncSetAttribute(tn_gemm_kernel<TN_F1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
             cudaSuccess ||
         cudaFuncSetAttribute(tn_gemm_kernel<TN_F2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(tn_gemm_kernel<TN_F1G>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
             cudaSuccess)
         return MOP_ERR_CUDA;
     return MOP_OK;
@@ -346,6 +401,24 @@ inline mop_status tn_up_swiglu(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, in
     g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
     p->prof->begin("gemm_up_swiglu", st);
     tn_gemm_kernel<TN_F1><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mXp, g);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+// Up-projection + SwiGLU reading its token rows straight from the unpermuted x (no Xp, no stash).
+inline mop_status tn_up_swiglu_gather(TcPlan* p, const bf16* x, const TcFwdArgs& a, int32_t* tiles, int32_t* status,
+                                      cudaStream_t st) {
+    const mop_moe_shape& s = p->s;
+    CUtensorMap mX, mWg, mWu;
+    if (!tc_map_2d(p, &mX, x, s.T, s.d, 1) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1) ||
+        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1))
+        return MOP_ERR_CUDA;
+    TnArgs g = tn_base_args(tiles, status);
+    g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
+    g.row_src = a.row_src; g.topk = s.k;
+    g.ep.out0 = a.H; g.ep.ldo = s.f; g.ep.M_total = s.T * s.k;
+    p->prof->begin("gemm_up_swiglu_gather", st);
+    tn_gemm_kernel<TN_F1G><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mX, g);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }

@@ -367,8 +367,8 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
 mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, int32_t* counts, int32_t* offsets,
                            int32_t* perm_row, int32_t* row_src, void* Xp, void* stream) {
     if (!c) return MOP_ERR_INVALID_ARG;
-    REQ_PTR_T(x); REQ_PTR_T(topk_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR_T(perm_row); REQ_PTR_T(row_src);
-    REQ_PTR_T(Xp);
+    REQ_PTR_T(topk_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR_T(perm_row); REQ_PTR_T(row_src);
+    if (Xp) { REQ_PTR_T(x); REQ_PTR_T(Xp); }   // Xp == NULL: tables only, for the gathering forward
     const mop_moe_shape& s = c->s;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MOP_ERR_CUDA;
@@ -391,6 +391,7 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
            perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, perm_row,
                                                                                         row_src, M, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
+    if (!Xp) return MOP_OK;
     const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
     LAUNCH(c, "permute_scatter_rows", st,
            scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row,
@@ -482,6 +483,28 @@ mop_status mop_moe_expert_ffn_fwd(mop_ctx* c, const void* Xp, const int32_t* off
     h.offsets = offsets; h.ragged_k = 0; h.N = s.d; h.Kfix = s.f; h.npairs = 1; h.epi = EPI_GATE;
     h.ep.out0 = static_cast<bf16*>(Yp); h.ep.gate = topk_gate; h.ep.row_src = row_src; h.ep.ldo = s.d; h.ep.M_total = M;
     return launch_scalar(c, "scalar_down_gate", h, st);
+}
+
+mop_status mop_moe_expert_ffn_fwd_gather(mop_ctx* c, const void* x, const int32_t* offsets, const int32_t* row_src,
+                                         const float* topk_gate, const void* W_gate, const void* W_up,
+                                         const void* W_down, void* H, void* Yp, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    REQ_PTR_T(x); REQ_PTR(offsets); REQ_PTR_T(row_src); REQ_PTR_T(topk_gate); REQ_PTR(W_gate); REQ_PTR(W_up);
+    REQ_PTR(W_down); REQ_PTR_T(H); REQ_PTR_T(Yp);
+    if (!use_tensor(c)) return MOP_ERR_UNSUPPORTED;   // the gather is a TMA feature of the tensor-core path
+    const mop_moe_shape& s = c->s;
+    if (s.T == 0) return MOP_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    TcFwdArgs a{};
+    a.x_gather = static_cast<const bf16*>(x); a.offsets = offsets; a.row_src = row_src; a.gate = topk_gate;
+    a.W_gate = static_cast<const bf16*>(W_gate); a.W_up = static_cast<const bf16*>(W_up);
+    a.W_down = static_cast<const bf16*>(W_down);
+    a.H = static_cast<bf16*>(H); a.Yp = static_cast<bf16*>(Yp);
+    int n = 0;
+    mop_status r = tc_ffn_fwd(&c->plan, a, c->tiles, c->status, static_cast<cudaStream_t>(stream), &n);
+    c->launches += n;
+    return r;
 }
 
 mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, const void* G_save,

@@ -4,6 +4,8 @@ Integers (top-k indices, counts, offsets, permutation) must match bit for bit.  
 Frobenius error <= 1e-2 against the oracle's exact mode and max-abs error <= 2e-2 against its
 declared-rounding mode (bf16 roundings at the tensors the interface declares bf16), per tensor.
 """
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -124,6 +126,45 @@ def test_two_cta_schedules_match_oracle_and_the_one_cta_kernel(path):
     _, _, _, ref = run(w, binding.GEMM_TENSOR_1CTA)
     for n in ("H", "Yp", "Y", "dX", "dgate", "dW_gate", "dW_up", "dW_down"):   # same accumulation order
         assert torch.equal(getattr(buf, n), getattr(ref, n)), n
+
+
+GATHER = [
+    synth.small("c3_trillion", T=200, d=256, E=40, k=8, f=128, seed=41),      # 40 rows per expert: one ragged tile each
+    synth.small("c2_mid", T=1500, d=256, E=6, k=2, f=320, seed=42),           # 500 rows per expert: two tiles
+    synth.small("c4_skew", T=1024, d=192, E=16, k=4, f=192, seed=43),         # skewed counts, hot and empty experts
+    synth.small("c1_tiny", T=3, d=64, E=5, k=1, f=64, seed=44),               # fewer rows than experts
+]
+
+
+@pytest.mark.parametrize("w", GATHER, ids=lambda w: f"{w.name}-T{w.T}d{w.d}E{w.E}k{w.k}f{w.f}")
+def test_gathering_forward_matches_oracle_and_the_permuting_forward(w):
+    host = synth.make_inputs(w, "cpu")
+    inp = to_dev(host)
+    ctx = binding.context_for(w, backward=False)
+    buf = binding.LayerBuffers(w)
+    buf.Xp.fill_(float("nan"))                       # the gathering form must not touch (or need) Xp
+    binding.forward(ctx, inp, buf, gather=True)
+    binding.mop_poll(ctx)
+    torch.cuda.synchronize()
+    assert torch.isnan(buf.Xp.float()).all()
+    xb, Wg, Wu, Wd = (synth.bits(host[n]) for n in ("x", "W_gate", "W_up", "W_down"))
+    idx, _ = oracle.route(xb, host["W_r"].numpy(), np_bias(host), w.k, w.score_fn, w.bias_mode)
+    assert np.array_equal(buf.idx.cpu().numpy(), idx)
+    gate = buf.gate.cpu().numpy()
+    Y_e = oracle.ffn_fwd(xb, idx, gate, Wg, Wu, Wd)
+    Y_d = oracle.ffn_fwd(xb, idx, gate, Wg, Wu, Wd, declared=True)
+    check_float("Y", buf.Y.float().cpu().numpy(), Y_e, Y_d)
+    _, _, _, ref = run(dataclasses.replace(w, backward=False), binding.GEMM_TENSOR_TN, host)
+    for n in ("H", "Yp", "Y"):                       # same tiles, same accumulation order
+        assert torch.equal(getattr(buf, n), getattr(ref, n)), n
+
+
+def test_gathering_forward_refuses_the_scalar_path():
+    w = synth.small("c1_tiny", T=77, d=72, E=5, k=2, f=40, seed=16)
+    host, inp, ctx, buf = run(w)
+    with pytest.raises(binding.MopError) as e:
+        binding.forward(ctx, inp, buf, gather=True)
+    assert e.value.code == 6
 
 
 def test_all_keys_equal_goes_to_lowest_ids_and_leaves_experts_empty():
