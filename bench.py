@@ -38,8 +38,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
 # (kernel, workload).  Filled from the summaries under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES: dict = {
-    # profiles/gemm_wgrad_gate_up_c5shape_E16.md: (66.0 MB read + 1820.9 MB written) at E = 16, x 384/16
-    ("gemm_wgrad_gate_up", "c5_train"): 24 * (66.024448e6 + 1.820895e9),
+    # profiles/dram_traffic_gemm_kernels.md: one-pass captures of the full-size launches
+    ("gemm_wgrad_gate_up", "c5_train"): 1477450496 + 45033558528,
+    ("gemm_up_swiglu", "c3_trillion"): 27582754048 + 536268032,
 }
 
 

@@ -131,6 +131,34 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         "[%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+// L2 eviction policies for the weight-gradient kernels: their fp32 output stream (tens of GB, never
+// re-read) would otherwise push the small operand set (an expert's rows, re-read by every tile of
+// that expert) out of L2 between uses.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 int z, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, "
+        "{%3, %4, %5}], [%2], %6;" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_3d_hint(const CUtensorMap* map, uint32_t src, int x, int y, int z,
+                                                  uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;" ::"l"(
+            map),
+        "r"(src), "r"(x), "r"(y), "r"(z), "l"(policy)
+        : "memory");
+}
 // shared -> global tile store (or fp32 add) of one box; completion is tracked by bulk groups
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map),
@@ -446,6 +474,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         // ===================================================================== TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool alive = true;
+            const uint64_t keep = l2_policy_evict_last();
+            (void)keep;
             // the next tile's descriptor is fetched one tile ahead so that its latency is hidden
             TileInfo nxt = decode_tile<KIND>(args, min((int)blockIdx.x, max(total_tiles - 1, 0)));
             for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
@@ -468,7 +498,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                         tma_load_2d(sA, ph ? &tmA1 : &tmA0, fb, k0, ti.row0);
                     } else {
                         // chunked map {64, rows, cols/64}: both 64-wide column chunks in one copy
-                        tma_load_3d(sA, &tmA0, fb, 0, ti.row0 + kb * TC_BK, ti.m0 >> 6);
+                        tma_load_3d_hint(sA, &tmA0, fb, 0, ti.row0 + kb * TC_BK, ti.m0 >> 6, keep);
                     }
                     if constexpr (!Tr::B_MN) {
                         tma_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0, n0, ti.e);
@@ -480,8 +510,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                             if constexpr (Tr::DUAL_B) tma_load_4d(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, k0, n0 >> 6, ti.e);
                         } else {
                             const int krow = ti.row0 + kb * TC_BK;
-                            tma_load_3d(sB, &tmB0, fb, 0, krow, n0 >> 6);
-                            if constexpr (Tr::DUAL_B) tma_load_3d(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, krow, n0 >> 6);
+                            tma_load_3d_hint(sB, &tmB0, fb, 0, krow, n0 >> 6, keep);
+                            if constexpr (Tr::DUAL_B) tma_load_3d_hint(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, krow, n0 >> 6, keep);
                         }
                     }
                     if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
@@ -595,6 +625,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 uint8_t* gbase = smem + TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + half * 32768;
                 const CUtensorMap* mo = (Tr::DUAL_B && half) ? &tmO1 : &tmO0;
                 const bool issuer = (quarter == 0 && lane == 0);
+                const uint64_t stream_out = l2_policy_evict_first();
                 const int gbar = 1 + half;               // named barrier of this half's 128 threads
                 float acc_b[32];
 #pragma unroll 1
@@ -621,7 +652,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                             const int gcol = n0 + (Tr::DUAL_B ? (col & 127) : col);
                             if (gcol < args.N) {
                                 if (args.ep.accumulate) tma_reduce_add_3d(mo, smem_u32(box), gcol, ti.m0, ti.e);
-                                else tma_store_3d(mo, smem_u32(box), gcol, ti.m0, ti.e);
+                                else tma_store_3d_hint(mo, smem_u32(box), gcol, ti.m0, ti.e, stream_out);
                             }
                             tma_store_commit();
                         }

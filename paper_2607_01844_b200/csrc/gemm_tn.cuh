@@ -67,7 +67,8 @@ __global__ void __launch_bounds__(1024) tn_build_ttiles_kernel(const int32_t* __
     }
     const int first = scan[e] - nt;
     const int sz = nt ? (((cnt + nt - 1) / nt + 15) & ~15) : 0;
-    for (int i = 0; i < nt; ++i) tiles[first + i] = make_int4(e, off + i * sz, min(sz, cnt - i * sz), 0);
+    // .w = position of the tile within its expert | number of tiles of the expert << 16
+    for (int i = 0; i < nt; ++i) tiles[first + i] = make_int4(e, off + i * sz, min(sz, cnt - i * sz), i | (nt << 16));
     if (e == 1023) *n_tiles = scan[1023];
 }
 
@@ -138,10 +139,21 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
     // work tile t -> token tile t / tiles_m (its expert, first row, rows) and weight-row tile t % tiles_m
     struct Tile { int e, row0, rows, nmma, mt; };
+    // Within an expert the token tiles vary fastest: the clusters that run at the same time on
+    // neighbouring work tiles then share one weight tile (the large operand) through L2.
     auto decode = [&](int t) {
-        const int4 m = __ldg(args.ttiles + t / args.tiles_m);
+        const int q = t / args.tiles_m;
+        int4 m = __ldg(args.ttiles + q);
+        const int nt = m.w >> 16;
         Tile ti;
-        ti.e = m.x; ti.row0 = m.y; ti.rows = m.z; ti.nmma = (m.z + 15) & ~15; ti.mt = t % args.tiles_m;
+        ti.mt = t % args.tiles_m;
+        if (nt > 1) {
+            const int first = q - (m.w & 0xffff);                 // first token tile of this expert
+            const int l = t - first * args.tiles_m;               // position among the expert's work tiles
+            ti.mt = l / nt;
+            m = __ldg(args.ttiles + first + l % nt);
+        }
+        ti.e = m.x; ti.row0 = m.y; ti.rows = m.z; ti.nmma = (m.z + 15) & ~15;
         return ti;
     };
 
