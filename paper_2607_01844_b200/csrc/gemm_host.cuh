@@ -148,7 +148,13 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
                                      launches)) != MOP_OK)
             return r;
     }
-    {   // B4: dXp = dG W_gate^T + dU W_up^T
+    if (p->fwd_tn & 4) {   // B4 on the tokens-on-N kernel
+        int32_t* ttiles = tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4);
+        if ((r = tn_build_tiles(p, a.offsets, ttiles, st)) != MOP_OK) return r;
+        ++*launches;
+        if ((r = tn_dgrad_gate_up(p, a, ttiles, status, st)) != MOP_OK) return r;
+        ++*launches;
+    } else {   // B4: dXp = dG W_gate^T + dU W_up^T
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.N = s.d;
         g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;

@@ -17,6 +17,8 @@
 //          single-GPU form of keeping only a fraction of the routed inputs live, Section 3.3).
 //          The TMA unit retires these 4-row copies far more slowly than one 128-row box (about
 //          60 ns each on B200), so this form trades time for memory and is opt-in.
+//   TN_B4  dXp^T = W_gate[e] dG^T + W_up[e] dU^T: the weights are read K-major ([E, d, f] as it
+//          lies in memory, rows of d on M), two K phases into one accumulator, dXp token-major.
 //
 // The epilogue transposes 32 x 32 blocks through shared memory so that global stores are 64-byte
 // row segments.  Barrier protocol, bounded waits and teardown as in the pair kernel.
@@ -25,7 +27,7 @@
 
 namespace mop {
 
-enum : int { TN_F1 = 0, TN_F2 = 1, TN_F1G = 2 };
+enum : int { TN_F1 = 0, TN_F2 = 1, TN_F1G = 2, TN_B4 = 3 };
 
 constexpr int TN_STAGES = 5;
 constexpr int TN_A_BYTES = 128 * TC_BK * 2;          // 16 KiB: this CTA's 128 weight rows
@@ -101,7 +103,7 @@ __device__ __forceinline__ uint16_t bf16_bits(float v) {
 template <int KIND>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TN_THREADS, 1)
 tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
-               const __grid_constant__ CUtensorMap tmB, const TnArgs args) {
+               const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmB1, const TnArgs args) {
     constexpr int S = TN_STAGES;
     extern __shared__ uint8_t tc_smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -127,6 +129,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB);
         if (KIND != TN_F2) tma_prefetch_desc(&tmA1);
+        if (KIND == TN_B4) tma_prefetch_desc(&tmB1);
     }
     if (warp == 1) tmem2_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
@@ -136,6 +139,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
 
     const int total_tiles = (*args.n_ttiles) * args.tiles_m;
+    const int nkb = (KIND == TN_B4 ? 2 : 1) * args.kblocks;   // K blocks per tile (B4: two phases)
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
     // work tile t -> token tile t / tiles_m (its expert, first row, rows) and weight-row tile t % tiles_m
     struct Tile { int e, row0, rows, nmma, mt; };
@@ -205,7 +209,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                 const int nbox = (half + TN_BOX_ROWS - 1) / TN_BOX_ROWS;
                 const int brow0 = ti.row0 + (int)rank * half;
                 const uint32_t tx = 2u * (TN_A_BYTES + (uint32_t)nbox * TN_BOX_ROWS * 128u);
-                for (int kb = 0; kb < args.kblocks; ++kb) {
+                for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) {
                         alive = false; break;
                     }
@@ -213,7 +217,17 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     if (leader) mbar_expect_tx(full_bar(stage), tx);
                     const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
                     const uint32_t sB = sA + TN_A_BYTES;
-                    const int k0 = kb * TC_BK;
+                    const int ph = (KIND == TN_B4 && kb >= args.kblocks) ? 1 : 0;   // B4: gate phase, then up phase
+                    const int k0 = (kb - ph * args.kblocks) * TC_BK;
+                    if constexpr (KIND == TN_B4) {
+                        // K-major weights: this CTA's 128 rows of d, 64 columns of f, one box
+                        const int m0 = ti.mt * 256 + 128 * (int)rank;
+                        tma2_load_3d(sA, ph ? &tmA1 : &tmA0, fb, k0, m0, ti.e);
+                        for (int b = 0; b < nbox; ++b)
+                            tma2_load_2d(sB + b * TN_BOX_ROWS * 128, ph ? &tmB1 : &tmB, fb, k0, brow0 + b * TN_BOX_ROWS);
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     if constexpr (KIND != TN_F2) {
                         // 64 gate columns, then the 64 matching up columns (N-major weights [E, d, f])
                         const int f0 = ti.mt * 128 + 64 * (int)rank;
@@ -237,8 +251,9 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
                 const Tile ti = nxt;
                 if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
-                // A is M-major (N-major weights), B is K-major; M = 256 over the pair, N = this tile's tokens
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) |
+                // A is M-major (N-major weights; K-major for B4), B is K-major; M = 256 over the pair,
+                // N = this tile's tokens
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((KIND == TN_B4 ? 0u : 1u) << 15) |
                                        ((uint32_t)(ti.nmma >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
                 const int buf = it & 1;
                 const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
@@ -246,7 +261,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * 256;
-                for (int kb = 0; kb < args.kblocks; ++kb) {
+                for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait_warp(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL, lane)) {
                         alive = false; break;
                     }
@@ -255,9 +270,11 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     const uint32_t sB = sA + TN_A_BYTES;
                     if (lane == 0) {
 #pragma unroll
-                        for (int k4 = 0; k4 < TC_BK / 16; ++k4)
-                            umma2_bf16(d_tmem, smem_desc(sA + k4 * 2048, TC_CHUNK_BYTES, 1024),
-                                       smem_desc(sB + k4 * 32, 0, 1024), idesc, (kb | k4) != 0 ? 1u : 0u);
+                        for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
+                            const uint64_t da = (KIND == TN_B4) ? smem_desc(sA + k4 * 32, 0, 1024)
+                                                                : smem_desc(sA + k4 * 2048, TC_CHUNK_BYTES, 1024);
+                            umma2_bf16(d_tmem, da, smem_desc(sB + k4 * 32, 0, 1024), idesc, (kb | k4) != 0 ? 1u : 0u);
+                        }
                         umma2_commit_both(empty_bar(stage));
                     }
                     __syncwarp();
@@ -285,7 +302,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256;
             float v[32];
 
-            if constexpr (KIND != TN_F2) {
+            if constexpr (KIND == TN_F1 || KIND == TN_F1G) {
                 // lanes 0..63 of the CTA hold gate rows, lanes 64..127 the matching up rows
                 const bool is_up = quarter >= 2;
                 const int fcol = ti.mt * 128 + 64 * (int)rank + 32 * (quarter & 1);   // first f of this warp
@@ -340,8 +357,10 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     tmem_ld32(taddr + c, v);
                     const int rows_left = ti.rows - c;
                     // gate of token (c + lane), handed round by shuffle
-                    float gmine = 0.0f;
-                    if (lane < rows_left) gmine = args.ep.gate[args.ep.row_src[ti.row0 + c + lane]];
+                    float gmine = (KIND == TN_B4) ? 1.0f : 0.0f;
+                    if constexpr (KIND == TN_F2) {
+                        if (lane < rows_left) gmine = args.ep.gate[args.ep.row_src[ti.row0 + c + lane]];
+                    }
 #pragma unroll
                     for (int tk = 0; tk < 32; ++tk) {
                         const float g = __shfl_sync(0xffffffffu, gmine, tk);
@@ -380,6 +399,8 @@ inline mop_status tn_init() {
         cudaFuncSetAttribute(tn_gemm_kernel<TN_F2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
             cudaSuccess ||
         cudaFuncSetAttribute(tn_gemm_kernel<TN_F1G>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(tn_gemm_kernel<TN_B4>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
             cudaSuccess)
         return MOP_ERR_CUDA;
     return MOP_OK;
@@ -412,7 +433,7 @@ inline mop_status tn_up_swiglu(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, in
     g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
     g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
     p->prof->begin("gemm_up_swiglu", st);
-    tn_gemm_kernel<TN_F1><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mXp, g);
+    tn_gemm_kernel<TN_F1><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mXp, mXp, g);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
@@ -430,7 +451,7 @@ inline mop_status tn_up_swiglu_gather(TcPlan* p, const bf16* x, const TcFwdArgs&
     g.row_src = a.row_src; g.topk = s.k;
     g.ep.out0 = a.H; g.ep.ldo = s.f; g.ep.M_total = s.T * s.k;
     p->prof->begin("gemm_up_swiglu_gather", st);
-    tn_gemm_kernel<TN_F1G><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mX, g);
+    tn_gemm_kernel<TN_F1G><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mX, mX, g);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
@@ -446,7 +467,24 @@ inline mop_status tn_down_gate(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, in
     g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.Mw = s.d;
     g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
     p->prof->begin("gemm_down_gate", st);
-    tn_gemm_kernel<TN_F2><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWd, mWd, mH, g);
+    tn_gemm_kernel<TN_F2><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWd, mWd, mH, mH, g);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+// Data gradient of the up-projection on the tokens-on-N kernel: dXp = dG W_gate^T + dU W_up^T.
+inline mop_status tn_dgrad_gate_up(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
+    const mop_moe_shape& s = p->s;
+    const uint64_t M = (uint64_t)s.T * s.k;
+    CUtensorMap mWg, mWu, mdG, mdU;
+    if (!tc_map_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 128) || !tc_map_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 128) ||
+        !tc_map_2d(p, &mdG, a.dG, M, s.f, TN_BOX_ROWS) || !tc_map_2d(p, &mdU, a.dU, M, s.f, TN_BOX_ROWS))
+        return MOP_ERR_CUDA;
+    TnArgs g = tn_base_args(tiles, status);
+    g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.Mw = s.d;
+    g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
+    p->prof->begin("gemm_dgrad_gate_up", st);
+    tn_gemm_kernel<TN_B4><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mdG, mdU, g);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }

@@ -285,9 +285,10 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         // up-projection wins when the K loop is long enough to hide its heavier epilogue (d >= 4096).
         c->plan.fwd_tn = 0;
         if (c->sm_count >= 2) {
-            if (shape->gemm_path == MOP_GEMM_TENSOR_TN) c->plan.fwd_tn = 3;
+            // bit 2: the data gradient of the up-projection on the same kernel
+            if (shape->gemm_path == MOP_GEMM_TENSOR_TN) c->plan.fwd_tn = 7;
             else if (shape->gemm_path == MOP_GEMM_AUTO || shape->gemm_path == MOP_GEMM_TENSOR)
-                c->plan.fwd_tn = 2 | (shape->d >= 4096 ? 1 : 0);
+                c->plan.fwd_tn = 4 | 2 | (shape->d >= 4096 ? 1 : 0);
         }
     }
     *out = c;
