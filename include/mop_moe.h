@@ -69,7 +69,8 @@ typedef struct {
                               recompute G, U, H in the backward (activation checkpointing) */
     int32_t dw_accumulate; /* 0: dW is overwritten (empty experts get zeros); 1: dW += */
     int32_t gemm_path;     /* mop_gemm_path; AUTO = tensor cores when the shape allows */
-    int32_t host_io;       /* 1: the context also holds the activations of mop_moe_forward_host */
+    int32_t host_io;       /* 1: the context also holds the activations of the host-buffer entry points;
+                              2: and a second slot of every buffer a copy touches, for the *_async forms */
 } mop_moe_shape;
 
 /* Create / destroy a context on `device` (a CUDA ordinal).  mop_create allocates the
@@ -187,6 +188,24 @@ mop_status mop_moe_route_bwd(mop_ctx* ctx, const float* logits, const float* bia
 mop_status mop_moe_forward_host(mop_ctx* ctx, const void* x_host, const float* W_r, const float* bias,
                                 const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
                                 int32_t* idx_host, float* gate_host, void* stream);
+
+/* Pipelined forms of the two host-buffer entry points (the paper has no counterpart: it never
+ * leaves the device).  A call enqueues one step and returns without waiting: its inputs are copied
+ * on a copy stream while the previous step computes on `stream`, and its results are copied out on
+ * an output stream while the next step computes.  The context double-buffers what the copies
+ * touch (host_io = 2).  Host buffers must be pinned for the copies to overlap, must stay valid and
+ * untouched until mop_host_drain returns, and output buffers of the last TWO calls must be
+ * distinct only if the caller reads them before draining.  mop_host_drain makes `stream` wait for
+ * every outstanding copy and synchronises it; errors of the kernels surface through mop_poll.
+ * Arguments as in the synchronous forms; results are bit-identical to them. */
+mop_status mop_moe_forward_host_async(mop_ctx* ctx, const void* x_host, const float* W_r, const float* bias,
+                                      const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
+                                      int32_t* idx_host, float* gate_host, void* stream);
+mop_status mop_moe_train_step_host_async(mop_ctx* ctx, const void* x_host, const void* dY_host, const float* W_r,
+                                         const float* bias, const void* W_gate, const void* W_up,
+                                         const void* W_down, void* Y_host, void* dX_host, float* dgate_host,
+                                         float* dW_gate, float* dW_up, float* dW_down, void* stream);
+mop_status mop_host_drain(mop_ctx* ctx, void* stream);
 
 /* Whole training step of the layer with HOST activations: copies x and dY in, runs route,
  * permute, expert_ffn_fwd (keeping G, U), combine and expert_ffn_bwd on `stream`, copies Y, dX

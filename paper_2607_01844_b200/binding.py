@@ -60,6 +60,9 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_combine.argtypes = [_P] * 5
         L.mop_moe_expert_ffn_bwd.argtypes = [_P] * 19
         L.mop_moe_forward_host.argtypes = [_P] * 11
+        L.mop_moe_forward_host_async.argtypes = [_P] * 11
+        L.mop_moe_train_step_host_async.argtypes = [_P] * 15
+        L.mop_host_drain.argtypes = [_P] * 2
         L.mop_moe_route_bwd.argtypes = [_P] * 14
         L.mop_moe_train_step_host.argtypes = [_P] * 15
         L.mop_moe_permute_static.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 4 + [_P] * 8
@@ -193,6 +196,29 @@ def mop_moe_train_step_host(ctx, x_host, dY_host, W_r, bias, W_gate, W_up, W_dow
            lib().mop_moe_train_step_host(ctx.handle, _ptr(x_host), _ptr(dY_host), _ptr(W_r), _ptr(bias), _ptr(W_gate),
                                          _ptr(W_up), _ptr(W_down), _ptr(Y_host), _ptr(dX_host), _ptr(dgate_host),
                                          _ptr(dW_gate), _ptr(dW_up), _ptr(dW_down), _stream(stream)))
+
+
+def mop_moe_forward_host_async(ctx, x_host, W_r, bias, W_gate, W_up, W_down, Y_host, idx_host=None, gate_host=None,
+                               stream=None):
+    """Enqueues one forward on PINNED host tensors and returns; results are valid after mop_host_drain."""
+    _check("mop_moe_forward_host_async",
+           lib().mop_moe_forward_host_async(ctx.handle, _ptr(x_host), _ptr(W_r), _ptr(bias), _ptr(W_gate),
+                                            _ptr(W_up), _ptr(W_down), _ptr(Y_host), _ptr(idx_host), _ptr(gate_host),
+                                            _stream(stream)))
+
+
+def mop_moe_train_step_host_async(ctx, x_host, dY_host, W_r, bias, W_gate, W_up, W_down, Y_host, dX_host, dgate_host,
+                                  dW_gate, dW_up, dW_down, stream=None):
+    """Enqueues one training step on PINNED host tensors and returns; results are valid after mop_host_drain."""
+    _check("mop_moe_train_step_host_async",
+           lib().mop_moe_train_step_host_async(ctx.handle, _ptr(x_host), _ptr(dY_host), _ptr(W_r), _ptr(bias),
+                                               _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(Y_host), _ptr(dX_host),
+                                               _ptr(dgate_host), _ptr(dW_gate), _ptr(dW_up), _ptr(dW_down),
+                                               _stream(stream)))
+
+
+def mop_host_drain(ctx, stream=None):
+    _check("mop_host_drain", lib().mop_host_drain(ctx.handle, _stream(stream)))
 
 
 def mop_moe_permute_static(device, T, d, E, k, x, topk_idx, counts, offsets, perm_row, row_src, Xp, stream=None):

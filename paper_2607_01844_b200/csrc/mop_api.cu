@@ -40,6 +40,14 @@ struct mop_ctx {
     float *hgate, *hdgate;
     cudaStream_t copy_stream;            // host-buffer entry points: copies that overlap the kernels
     cudaEvent_t ev_in, ev_mid, ev_out;
+    // pipelined host entry points (host_io = 2): the second set of the buffers that copies touch,
+    // a stream for device-to-host copies, and per-slot events
+    bf16 *px[2], *pY[2], *pdY[2], *pdX[2];
+    int32_t* pidx[2];
+    float *pgate[2], *pdgate[2];
+    cudaStream_t out_stream;
+    cudaEvent_t ev_x[2], ev_dy[2], ev_fwd[2], ev_done[2], ev_drained[2];
+    uint64_t host_steps;
     TcPlan plan;
     Profiler prof;
 };
@@ -52,6 +60,7 @@ struct Layout {
     size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT, rG, rU, rH;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
     size_t hG, hU, hdY, hdX, hdgate;
+    size_t qx, qY, qidx, qgate, qdY, qdX, qdgate;   // second slot of the pipelined host entry points
     size_t total;
 };
 
@@ -102,6 +111,17 @@ Layout make_layout(const mop_moe_shape& s) {
             L.hdX = take(T * d * 2);
             L.hdgate = take(M * 4);
         }
+        if (s.host_io == 2) {
+            L.qx = take(T * d * 2);
+            L.qY = take(T * d * 2);
+            L.qidx = take(M * 4);
+            L.qgate = take(M * 4);
+            if (s.with_backward) {
+                L.qdY = take(T * d * 2);
+                L.qdX = take(T * d * 2);
+                L.qdgate = take(M * 4);
+            }
+        }
     }
     L.total = o;
     return L;
@@ -119,6 +139,7 @@ mop_status check_shape(const mop_moe_shape* s) {
     if (s->E > SEL_MAX_E || s->k > 32) return MOP_ERR_SHAPE;
     if ((long long)s->T * s->d >= (1ll << 40) || (long long)s->d * s->f >= (1ll << 31)) return MOP_ERR_SHAPE;
     if (s->d % 8 || s->f % 8) return MOP_ERR_ALIGN;
+    if (s->host_io < 0 || s->host_io > 2) return MOP_ERR_INVALID_ARG;
     return MOP_OK;
 }
 
@@ -265,7 +286,32 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
             c->hdgate = reinterpret_cast<float*>(w + L.hdgate);
         }
     }
+    if (shape->host_io) {
+        c->px[0] = c->hx; c->pY[0] = c->hY; c->pidx[0] = c->hidx; c->pgate[0] = c->hgate;
+        c->pdY[0] = c->hdY; c->pdX[0] = c->hdX; c->pdgate[0] = c->hdgate;
+    }
+    if (shape->host_io == 2) {
+        c->px[1] = reinterpret_cast<bf16*>(w + L.qx);
+        c->pY[1] = reinterpret_cast<bf16*>(w + L.qY);
+        c->pidx[1] = reinterpret_cast<int32_t*>(w + L.qidx);
+        c->pgate[1] = reinterpret_cast<float*>(w + L.qgate);
+        if (shape->with_backward) {
+            c->pdY[1] = reinterpret_cast<bf16*>(w + L.qdY);
+            c->pdX[1] = reinterpret_cast<bf16*>(w + L.qdX);
+            c->pdgate[1] = reinterpret_cast<float*>(w + L.qdgate);
+        }
+    }
     if (cudaMemset(c->status, 0, 256) != cudaSuccess) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
+    if (shape->host_io == 2) {
+        bool ok = cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; i < 2 && ok; ++i)
+            ok = cudaEventCreateWithFlags(&c->ev_x[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_dy[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_fwd[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->ev_drained[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
+    }
     if (shape->host_io) {
         if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_in, cudaEventDisableTiming) != cudaSuccess ||
@@ -305,6 +351,13 @@ void mop_destroy(mop_ctx* c) {
     if (c->s.host_io) {
         cudaStreamDestroy(c->copy_stream);
         cudaEventDestroy(c->ev_in); cudaEventDestroy(c->ev_mid); cudaEventDestroy(c->ev_out);
+    }
+    if (c->s.host_io == 2) {
+        cudaStreamDestroy(c->out_stream);
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(c->ev_x[i]); cudaEventDestroy(c->ev_dy[i]); cudaEventDestroy(c->ev_fwd[i]);
+            cudaEventDestroy(c->ev_done[i]); cudaEventDestroy(c->ev_drained[i]);
+        }
     }
     cudaFree(c->ws);
     delete c;
@@ -691,6 +744,104 @@ mop_status step_host(mop_ctx* c, const void* x_host, const void* dY_host, const 
     return MOP_OK;
 }
 }  // namespace
+
+namespace {
+// One step on host buffers WITHOUT waiting for it: step i's inputs come in on the copy stream while
+// step i-1 computes, its results leave on the output stream while step i+1 computes.  Two slots of
+// every buffer a copy touches; per-slot events order the three streams:
+//   copy stream   : [slot free: step i-2 computed] -> x, dY in          -> ev_x, ev_dy
+//   caller stream : [ev_x] [slot's results of step i-2 copied out] forward -> ev_fwd, [ev_dy] backward -> ev_done
+//   output stream : [ev_fwd] Y, idx, gate out; [ev_done] dX, dgate out  -> ev_drained
+mop_status step_host_pipelined(mop_ctx* c, const void* x_host, const void* dY_host, const float* W_r,
+                               const float* bias, const void* W_gate, const void* W_up, const void* W_down,
+                               void* Y_host, int32_t* idx_host, float* gate_host, void* dX_host, float* dgate_host,
+                               float* dW_gate, float* dW_up, float* dW_down, void* stream) {
+    const mop_moe_shape& s = c->s;
+    const bool bwd = dY_host != nullptr;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream), in = c->copy_stream, out = c->out_stream;
+    const size_t M = (size_t)s.T * s.k, xb = (size_t)s.T * s.d * 2;
+    const int q = (int)(c->host_steps++ & 1);
+    if (s.T > 0) {
+        CUDA_OK(cudaStreamWaitEvent(in, c->ev_done[q], 0));       // step i-2 no longer reads this slot's inputs
+        CUDA_OK(cudaMemcpyAsync(c->px[q], x_host, xb, cudaMemcpyHostToDevice, in));
+        CUDA_OK(cudaEventRecord(c->ev_x[q], in));
+        if (bwd) {
+            CUDA_OK(cudaMemcpyAsync(c->pdY[q], dY_host, xb, cudaMemcpyHostToDevice, in));
+            CUDA_OK(cudaEventRecord(c->ev_dy[q], in));
+        }
+        CUDA_OK(cudaStreamWaitEvent(st, c->ev_x[q], 0));
+        CUDA_OK(cudaStreamWaitEvent(st, c->ev_drained[q], 0));    // step i-2's results have left this slot
+    }
+    mop_status r;
+    if ((r = mop_moe_route(c, c->px[q], W_r, bias, c->pidx[q], c->pgate[q], nullptr, stream)) != MOP_OK) return r;
+    if ((r = mop_moe_permute(c, c->px[q], c->pidx[q], c->hcounts, c->hoffsets, c->hperm, c->hsrc, c->hXp, stream)) !=
+        MOP_OK)
+        return r;
+    if ((r = mop_moe_expert_ffn_fwd(c, c->hXp, c->hoffsets, c->hsrc, c->pgate[q], W_gate, W_up, W_down,
+                                    bwd ? c->hG : nullptr, bwd ? c->hU : nullptr, c->hH, c->hYp, stream)) != MOP_OK)
+        return r;
+    if ((r = mop_moe_combine(c, c->hYp, c->hperm, c->pY[q], stream)) != MOP_OK) return r;
+    if (s.T > 0) {
+        CUDA_OK(cudaEventRecord(c->ev_fwd[q], st));
+        CUDA_OK(cudaStreamWaitEvent(out, c->ev_fwd[q], 0));
+        CUDA_OK(cudaMemcpyAsync(Y_host, c->pY[q], xb, cudaMemcpyDeviceToHost, out));
+        if (idx_host) CUDA_OK(cudaMemcpyAsync(idx_host, c->pidx[q], M * 4, cudaMemcpyDeviceToHost, out));
+        if (gate_host) CUDA_OK(cudaMemcpyAsync(gate_host, c->pgate[q], M * 4, cudaMemcpyDeviceToHost, out));
+    }
+    if (bwd) {
+        if (s.T > 0) CUDA_OK(cudaStreamWaitEvent(st, c->ev_dy[q], 0));
+        if ((r = mop_moe_expert_ffn_bwd(c, c->pdY[q], c->hXp, c->hG, c->hU, c->hH, c->hoffsets, c->hperm, c->hsrc,
+                                        c->pgate[q], W_gate, W_up, W_down, c->pdX[q], dW_gate, dW_up, dW_down,
+                                        c->pdgate[q], stream)) != MOP_OK)
+            return r;
+    }
+    if (s.T > 0) {
+        CUDA_OK(cudaEventRecord(c->ev_done[q], st));
+        if (bwd) {
+            CUDA_OK(cudaStreamWaitEvent(out, c->ev_done[q], 0));
+            CUDA_OK(cudaMemcpyAsync(dX_host, c->pdX[q], xb, cudaMemcpyDeviceToHost, out));
+            if (dgate_host) CUDA_OK(cudaMemcpyAsync(dgate_host, c->pdgate[q], M * 4, cudaMemcpyDeviceToHost, out));
+        }
+        CUDA_OK(cudaEventRecord(c->ev_drained[q], out));
+    }
+    return MOP_OK;
+}
+}  // namespace
+
+mop_status mop_moe_forward_host_async(mop_ctx* c, const void* x_host, const float* W_r, const float* bias,
+                                      const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
+                                      int32_t* idx_host, float* gate_host, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (c->s.T > 0 && (!x_host || !Y_host)) return MOP_ERR_INVALID_ARG;
+    if (c->s.host_io != 2) return MOP_ERR_UNSUPPORTED;
+    return step_host_pipelined(c, x_host, nullptr, W_r, bias, W_gate, W_up, W_down, Y_host, idx_host, gate_host,
+                               nullptr, nullptr, nullptr, nullptr, nullptr, stream);
+}
+
+mop_status mop_moe_train_step_host_async(mop_ctx* c, const void* x_host, const void* dY_host, const float* W_r,
+                                         const float* bias, const void* W_gate, const void* W_up, const void* W_down,
+                                         void* Y_host, void* dX_host, float* dgate_host, float* dW_gate,
+                                         float* dW_up, float* dW_down, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (c->s.T > 0 && (!x_host || !dY_host || !Y_host || !dX_host)) return MOP_ERR_INVALID_ARG;
+    if (c->s.host_io != 2 || !c->s.with_backward) return MOP_ERR_UNSUPPORTED;
+    if (c->s.T == 0 && !dY_host) dY_host = c;  // any non-null token: selects the backward branch
+    return step_host_pipelined(c, x_host, dY_host, W_r, bias, W_gate, W_up, W_down, Y_host, nullptr, nullptr,
+                               dX_host, dgate_host, dW_gate, dW_up, dW_down, stream);
+}
+
+mop_status mop_host_drain(mop_ctx* c, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (c->s.host_io != 2) return MOP_ERR_UNSUPPORTED;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int q = 0; q < 2; ++q) CUDA_OK(cudaStreamWaitEvent(st, c->ev_drained[q], 0));
+    CUDA_OK(cudaStreamSynchronize(st));
+    return MOP_OK;
+}
 
 mop_status mop_moe_forward_host(mop_ctx* c, const void* x_host, const float* W_r, const float* bias,
                                 const void* W_gate, const void* W_up, const void* W_down, void* Y_host,

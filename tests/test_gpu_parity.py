@@ -239,6 +239,64 @@ def test_forward_host_entry_point_matches_device_path():
     assert torch.equal(Yh, buf.Y.cpu()) and torch.equal(idxh, buf.idx.cpu()) and torch.equal(gh, buf.gate.cpu())
 
 
+@pytest.mark.parametrize("backward", [False, True], ids=["fwd", "train"])
+def test_pipelined_host_steps_match_the_device_path_step_by_step(backward):
+    """Five steps with different inputs in flight through the two slots; every step's results are its own."""
+    w = synth.small("c2_mid", T=300, d=128, E=8, k=2, f=192, seed=23, backward=backward)
+    steps = 5
+    hosts = [synth.make_inputs(dataclasses.replace(w, seed=100 + i), "cpu") for i in range(steps)]
+    weights = to_dev(hosts[0])                      # one set of weights, per-step activations
+    ctx = binding.context_for(w, host_io=2)
+    outs = []
+    for h in hosts:
+        o = {"x": h["x"].pin_memory(), "Y": torch.empty_like(h["x"]).pin_memory(),
+             "idx": torch.empty((w.T, w.k), dtype=torch.int32).pin_memory(),
+             "gate": torch.empty((w.T, w.k), dtype=torch.float32).pin_memory()}
+        if backward:
+            o["dY"] = h["dY"].pin_memory()
+            o["dX"] = torch.empty_like(h["x"]).pin_memory()
+            o["dgate"] = torch.empty((w.T, w.k), dtype=torch.float32).pin_memory()
+        outs.append(o)
+    dW = [torch.empty_like(weights[n], dtype=torch.float32) for n in ("W_gate", "W_up", "W_down")]
+    for o in outs:
+        if backward:
+            binding.mop_moe_train_step_host_async(ctx, o["x"], o["dY"], weights["W_r"], weights["bias"],
+                                                  weights["W_gate"], weights["W_up"], weights["W_down"], o["Y"],
+                                                  o["dX"], o["dgate"], *dW)
+        else:
+            binding.mop_moe_forward_host_async(ctx, o["x"], weights["W_r"], weights["bias"], weights["W_gate"],
+                                               weights["W_up"], weights["W_down"], o["Y"], o["idx"], o["gate"])
+    binding.mop_host_drain(ctx)
+    binding.mop_poll(ctx)
+    ref_ctx = binding.context_for(w)
+    for i, (h, o) in enumerate(zip(hosts, outs)):
+        inp = dict(weights)
+        inp["x"] = h["x"].cuda()
+        if backward:
+            inp["dY"] = h["dY"].cuda()
+        buf = binding.LayerBuffers(w)
+        binding.forward(ref_ctx, inp, buf)
+        if backward:
+            binding.backward(ref_ctx, inp, buf)
+        torch.cuda.synchronize()
+        assert torch.equal(o["Y"], buf.Y.cpu()), f"Y of step {i}"
+        if backward:
+            assert torch.equal(o["dX"], buf.dX.cpu()) and torch.equal(o["dgate"], buf.dgate.cpu()), f"step {i}"
+        else:
+            assert torch.equal(o["idx"], buf.idx.cpu()) and torch.equal(o["gate"], buf.gate.cpu()), f"step {i}"
+    if backward:   # dW holds the last step's gradients
+        for got, name in zip(dW, ("dW_gate", "dW_up", "dW_down")):
+            assert torch.equal(got, getattr(buf, name)), name
+
+
+def test_pipelined_host_entry_points_need_their_context_mode():
+    w = synth.small("c1_tiny", T=8, d=64, E=4, k=2, f=64, seed=24)
+    ctx = binding.context_for(w, host_io=True)
+    with pytest.raises(binding.MopError) as e:
+        binding.mop_host_drain(ctx)
+    assert e.value.code == 6
+
+
 ROUTER_BWD = [
     synth.small("c1_tiny", T=200, d=128, E=8, k=2, f=64, backward=True, seed=30),                       # softmax
     synth.small("c3_trillion", T=300, d=192, E=40, k=8, f=64, backward=True, seed=31),                  # sigmoid + post bias
