@@ -139,7 +139,16 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
         !tc_map_chunked_2d(p, &mXpA, a.Xp, M, s.d, 2) || !tc_map_chunked_2d(p, &mdGB, a.dG, M, s.f, 2) ||
         !tc_map_chunked_2d(p, &mdUB, a.dU, M, s.f, 2))
         return MOP_ERR_CUDA;
-    {   // B2: dHu = dYp W_down^T, SwiGLU backward epilogue
+    int32_t* ttiles = tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4);
+    if (p->fwd_tn & 12) {
+        if ((r = tn_build_tiles(p, a.offsets, ttiles, st)) != MOP_OK) return r;
+        ++*launches;
+    }
+    if (p->fwd_tn & 8) {   // B2 on the tokens-on-N kernel: one dgate partial per 32 columns of f
+        *ntile_part = ceil_div(s.f, 32);
+        if ((r = tn_dgrad_down(p, a, ttiles, status, st)) != MOP_OK) return r;
+        ++*launches;
+    } else {   // B2: dHu = dYp W_down^T, SwiGLU backward epilogue
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.f;
         g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
@@ -149,9 +158,6 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
             return r;
     }
     if (p->fwd_tn & 4) {   // B4 on the tokens-on-N kernel
-        int32_t* ttiles = tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4);
-        if ((r = tn_build_tiles(p, a.offsets, ttiles, st)) != MOP_OK) return r;
-        ++*launches;
         if ((r = tn_dgrad_gate_up(p, a, ttiles, status, st)) != MOP_OK) return r;
         ++*launches;
     } else {   // B4: dXp = dG W_gate^T + dU W_up^T

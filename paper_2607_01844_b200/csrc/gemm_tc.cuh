@@ -708,7 +708,7 @@ struct TcPlan {
     mop_moe_shape s;
     void* encode;   // cuTensorMapEncodeTiled
     int pairs;      // schedule of the token-row kinds (see gemm_host.cuh)
-    int fwd_tn;     // GEMMs on the tokens-on-N kernels: bit 0 up-projection, bit 1 down-projection, bit 2 dgrad of the up-projection
+    int fwd_tn;     // GEMMs on the tokens-on-N kernels: bit 0 up-projection, bit 1 down-projection, bit 2 dgrad of the up-projection, bit 3 dgrad of the down-projection
     Profiler* prof;
 };
 

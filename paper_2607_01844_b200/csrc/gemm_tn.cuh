@@ -19,6 +19,9 @@
 //          60 ns each on B200), so this form trades time for memory and is opt-in.
 //   TN_B4  dXp^T = W_gate[e] dG^T + W_up[e] dU^T: the weights are read K-major ([E, d, f] as it
 //          lies in memory, rows of d on M), two K phases into one accumulator, dXp token-major.
+//   TN_B2  dHu^T = W_down[e] dYp^T (weights K-major, rows of f on M); the epilogue turns each
+//          32 x 32 block token-major through shared memory and then runs the SwiGLU backward on
+//          16-byte runs of the stash: dG, dU, gate*H out, and one dgate partial per 32 columns of f.
 //
 // The epilogue transposes 32 x 32 blocks through shared memory so that global stores are 64-byte
 // row segments.  Barrier protocol, bounded waits and teardown as in the pair kernel.
@@ -27,7 +30,7 @@
 
 namespace mop {
 
-enum : int { TN_F1 = 0, TN_F2 = 1, TN_F1G = 2, TN_B4 = 3 };
+enum : int { TN_F1 = 0, TN_F2 = 1, TN_F1G = 2, TN_B4 = 3, TN_B2 = 4 };
 
 constexpr int TN_STAGES = 5;
 constexpr int TN_A_BYTES = 128 * TC_BK * 2;          // 16 KiB: this CTA's 128 weight rows
@@ -219,8 +222,8 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     const uint32_t sB = sA + TN_A_BYTES;
                     const int ph = (KIND == TN_B4 && kb >= args.kblocks) ? 1 : 0;   // B4: gate phase, then up phase
                     const int k0 = (kb - ph * args.kblocks) * TC_BK;
-                    if constexpr (KIND == TN_B4) {
-                        // K-major weights: this CTA's 128 rows of d, 64 columns of f, one box
+                    if constexpr (KIND == TN_B4 || KIND == TN_B2) {
+                        // K-major weights: this CTA's 128 weight rows, 64 columns of K, one box
                         const int m0 = ti.mt * 256 + 128 * (int)rank;
                         tma2_load_3d(sA, ph ? &tmA1 : &tmA0, fb, k0, m0, ti.e);
                         for (int b = 0; b < nbox; ++b)
@@ -253,7 +256,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                 if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
                 // A is M-major (N-major weights; K-major for B4), B is K-major; M = 256 over the pair,
                 // N = this tile's tokens
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((KIND == TN_B4 ? 0u : 1u) << 15) |
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((KIND == TN_B4 || KIND == TN_B2 ? 0u : 1u) << 15) |
                                        ((uint32_t)(ti.nmma >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
                 const int buf = it & 1;
                 const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
@@ -271,7 +274,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     if (lane == 0) {
 #pragma unroll
                         for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
-                            const uint64_t da = (KIND == TN_B4) ? smem_desc(sA + k4 * 32, 0, 1024)
+                            const uint64_t da = (KIND == TN_B4 || KIND == TN_B2) ? smem_desc(sA + k4 * 32, 0, 1024)
                                                                 : smem_desc(sA + k4 * 2048, TC_CHUNK_BYTES, 1024);
                             umma2_bf16(d_tmem, da, smem_desc(sB + k4 * 32, 0, 1024), idesc, (kb | k4) != 0 ? 1u : 0u);
                         }
@@ -348,6 +351,38 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     }
                     __syncwarp();
                 }
+            } else if constexpr (KIND == TN_B2) {
+                const int fcol = ti.mt * 256 + 128 * (int)rank + 32 * quarter;      // first f column of this warp
+                const bool f_ok = fcol < args.Mw;
+                float* fbuf = reinterpret_cast<float*>(wbuf);                       // 32 tokens x 33 fp32
+                const int part = lane & 3;
+#pragma unroll 1
+                for (int c = 0; c < ti.nmma; c += 32) {
+                    tmem_ld32(taddr + c, v);
+                    const int rows_left = ti.rows - c;
+#pragma unroll
+                    for (int tk = 0; tk < 32; ++tk) fbuf[tk * 33 + lane] = v[tk];
+                    __syncwarp();
+#pragma unroll 1
+                    for (int i = 0; i < 4; ++i) {
+                        const int tok = 8 * i + (lane >> 2);
+                        const bool ok = f_ok && tok < rows_left;
+                        float dot = 0.0f;
+                        if (ok) {
+                            const int row = ti.row0 + c + tok;
+                            const float gate = args.ep.gate[args.ep.row_src[row]];
+                            float dhu[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) dhu[j] = fbuf[tok * 33 + part * 8 + j];
+                            dot = epi_dh<8>(args.ep, row, fcol + part * 8, gate, dhu);
+                        }
+                        dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+                        dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+                        if (ok && part == 0)
+                            args.ep.part[(size_t)(fcol >> 5) * args.ep.M_total + ti.row0 + c + tok] = dot;
+                    }
+                    __syncwarp();
+                }
             } else {
                 const int mcol = ti.mt * 256 + 128 * (int)rank + 32 * quarter;      // first output column of this warp
                 const bool m_ok = mcol < args.Mw;
@@ -401,6 +436,8 @@ inline mop_status tn_init() {
         cudaFuncSetAttribute(tn_gemm_kernel<TN_F1G>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
             cudaSuccess ||
         cudaFuncSetAttribute(tn_gemm_kernel<TN_B4>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(tn_gemm_kernel<TN_B2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TN_SMEM_BYTES) !=
             cudaSuccess)
         return MOP_ERR_CUDA;
     return MOP_OK;
@@ -485,6 +522,24 @@ inline mop_status tn_dgrad_gate_up(TcPlan* p, const TcBwdArgs& a, int32_t* tiles
     g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
     p->prof->begin("gemm_dgrad_gate_up", st);
     tn_gemm_kernel<TN_B4><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mdG, mdU, g);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
+// Data gradient of the down-projection with the SwiGLU backward on the tokens-on-N kernel.
+// Writes one dgate partial per 32 columns of f (part[f / 32][row]).
+inline mop_status tn_dgrad_down(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
+    const mop_moe_shape& s = p->s;
+    const uint64_t M = (uint64_t)s.T * s.k;
+    CUtensorMap mWd, mdYp;
+    if (!tc_map_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 128) || !tc_map_2d(p, &mdYp, a.dYp, M, s.d, TN_BOX_ROWS))
+        return MOP_ERR_CUDA;
+    TnArgs g = tn_base_args(tiles, status);
+    g.tiles_m = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
+    g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
+    g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.part = a.part; g.ep.ldo = s.f; g.ep.M_total = (int)M;
+    p->prof->begin("gemm_dgrad_down_dswiglu", st);
+    tn_gemm_kernel<TN_B2><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWd, mWd, mdYp, mdYp, g);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }

@@ -65,7 +65,7 @@ struct Layout {
 };
 
 int perm_units(const mop_moe_shape& s) { return ceil_div(s.T * s.k, PERM_SEG); }
-int part_tiles(const mop_moe_shape& s) { return ceil_div(s.f, 64); }
+int part_tiles(const mop_moe_shape& s) { return ceil_div(s.f, 32); }
 
 Layout make_layout(const mop_moe_shape& s) {
     Layout L{};
@@ -331,10 +331,10 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         // up-projection wins when the K loop is long enough to hide its heavier epilogue (d >= 4096).
         c->plan.fwd_tn = 0;
         if (c->sm_count >= 2) {
-            // bit 2: the data gradient of the up-projection on the same kernel
-            if (shape->gemm_path == MOP_GEMM_TENSOR_TN) c->plan.fwd_tn = 7;
+            // bits 2, 3: the data gradients of the up- and down-projection on the same kernel
+            if (shape->gemm_path == MOP_GEMM_TENSOR_TN) c->plan.fwd_tn = 15;
             else if (shape->gemm_path == MOP_GEMM_AUTO || shape->gemm_path == MOP_GEMM_TENSOR)
-                c->plan.fwd_tn = 4 | 2 | (shape->d >= 4096 ? 1 : 0);
+                c->plan.fwd_tn = 8 | 4 | 2 | (shape->d >= 4096 ? 1 : 0);
         }
     }
     *out = c;
