@@ -36,7 +36,7 @@ typedef struct mop_ctx mop_ctx; /* opaque: shape, workspace, status word */
 typedef enum {
     MOP_OK = 0,
     MOP_ERR_INVALID_ARG = 1, /* null pointer, bad enum, k > E, ... */
-    MOP_ERR_SHAPE = 2,       /* sizes out of the supported range (T*k >= 2^31, E > 4096, ...) */
+    MOP_ERR_SHAPE = 2,       /* sizes out of the supported range (T*k >= 2^31, E > 1024, k > 32, ...) */
     MOP_ERR_ALIGN = 3,       /* pointer not 16-byte aligned, or d / f not a multiple of 8 */
     MOP_ERR_WORKSPACE = 4,   /* device allocation of the context's workspace failed */
     MOP_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed */

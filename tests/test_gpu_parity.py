@@ -228,6 +228,23 @@ def test_bad_arguments_return_codes():
     assert e.value.code == 1
 
 
+def test_largest_expert_count_and_routing_degree():
+    """E = 1024 and k = 32 are the limits of the selection kernel; most experts get zero to four rows."""
+    w = synth.small("c1_tiny", T=48, d=64, E=1024, k=32, f=64, backward=True, seed=27)
+    _, buf = check_layer(w, binding.GEMM_AUTO)
+    assert int((buf.counts == 0).sum()) > 0
+    w2 = synth.small("c3_trillion", T=40, d=64, E=1024, k=32, f=64, seed=28)      # sigmoid + bias at the limits
+    check_layer(w2, binding.GEMM_AUTO)
+
+
+def test_shapes_beyond_the_limits_are_refused():
+    for args, code in (((16, 64, 1025, 2, 64), 2), ((64, 64, 64, 33, 64), 2), ((16, 60, 4, 2, 64), 3),
+                       ((16, 64, 4, 2, 36), 3), ((-1, 64, 4, 2, 64), 1), ((16, 64, 0, 1, 64), 1)):
+        with pytest.raises(binding.MopError) as e:
+            binding.Context(*args)
+        assert e.value.code == code, args
+
+
 def test_forward_host_entry_point_matches_device_path():
     w = synth.small("c2_mid", T=256, d=128, E=8, k=2, f=192, seed=20)
     host, inp, _, buf = run(w)
