@@ -93,6 +93,10 @@ mop_status mop_selftest_wait_timeout(mop_ctx* ctx, int64_t limit_cycles, void* s
 /* Number of kernels launched through this context since it was created. */
 int64_t mop_launch_count(const mop_ctx* ctx);
 
+/* The device entry points below (route, permute, expert_ffn_fwd / _gather, combine, expert_ffn_bwd,
+ * route_bwd) only enqueue work on `stream`: no allocation, no synchronisation, no host read of device
+ * data.  A sequence of them may therefore be captured into a CUDA graph and replayed. */
+
 /* Router (Section 2.1: "a lightweight router that sends each token to its top-k experts").
  *   z[t,e]   = sum_i x[t,i] * W_r[i,e]: one fp32 fused multiply-add per i, i ascending.
  *   key      = z | sigmoid(z) + bias | z + bias       (score_fn, bias_mode)

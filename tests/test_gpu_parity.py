@@ -228,6 +228,28 @@ def test_bad_arguments_return_codes():
     assert e.value.code == 1
 
 
+def test_the_step_can_be_captured_into_a_cuda_graph_and_replayed():
+    """The device entry points allocate nothing and never synchronise, so a whole step captures."""
+    w = synth.small("c2_mid", T=512, d=256, E=16, k=4, f=192, backward=True, seed=29)
+    host, inp, ctx, ref = run(w)
+    buf = binding.LayerBuffers(w)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            binding.forward(ctx, inp, buf, side)
+            binding.backward(ctx, inp, buf, side)
+    torch.cuda.synchronize()
+    for _ in range(2):                                  # replays are steps of their own
+        for n in ("Y", "dX", "dgate", "dW_gate", "dW_up", "dW_down"):
+            getattr(buf, n).zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for n in ("idx", "gate", "Y", "dX", "dgate", "dW_gate", "dW_up", "dW_down"):
+            assert torch.equal(getattr(buf, n), getattr(ref, n)), n
+    binding.mop_poll(ctx)
+
+
 def test_largest_expert_count_and_routing_degree():
     """E = 1024 and k = 32 are the limits of the selection kernel; most experts get zero to four rows."""
     w = synth.small("c1_tiny", T=48, d=64, E=1024, k=32, f=64, backward=True, seed=27)
