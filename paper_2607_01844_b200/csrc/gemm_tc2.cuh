@@ -53,6 +53,14 @@ __device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* ma
         "%5, %6}], [%2];" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w)
         : "memory");
 }
+// the same copy with an L2 eviction policy
+__device__ __forceinline__ void tma2_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                  int z, int w, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], "
+        "[%1, {%3, %4, %5, %6}], [%2], %7;" ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ void tmem2_alloc(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
                  : "memory");

@@ -204,6 +204,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         // ===================================================================== TMA producer (both CTAs)
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0; bool alive = true;
+            const uint64_t pol_w = l2_policy_evict_last();
             Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
                 const Tile ti = nxt;
@@ -234,11 +235,11 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     if constexpr (KIND != TN_F2) {
                         // 64 gate columns, then the 64 matching up columns (N-major weights [E, d, f])
                         const int f0 = ti.mt * 128 + 64 * (int)rank;
-                        tma2_load_4d(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e);
-                        tma2_load_4d(sA + TC_CHUNK_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e);
+                        tma2_load_4d_hint(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e, pol_w);
+                        tma2_load_4d_hint(sA + TC_CHUNK_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e, pol_w);
                     } else {
                         const int m0 = ti.mt * 256 + 128 * (int)rank;
-                        tma2_load_4d(sA, &tmA0, fb, 0, k0, m0 >> 6, ti.e);   // two chunks in one copy
+                        tma2_load_4d_hint(sA, &tmA0, fb, 0, k0, m0 >> 6, ti.e, pol_w);   // two chunks in one copy
                     }
                     for (int b = 0; b < nbox; ++b)
                         tma2_load_2d(sB + b * TN_BOX_ROWS * 128, &tmB, fb, k0, brow0 + b * TN_BOX_ROWS);
