@@ -290,3 +290,25 @@ def vocab_loss(x_bits, W_bits, targets):
     m = Y.max(1)
     lse = m + np.log(np.exp(Y - m[:, None]).sum(1))
     return Y[np.arange(Y.shape[0]), t] - lse, lse
+
+
+def vocab_loss_bwd(x_bits, W_bits, targets, dloss, declared=False):
+    """Gradients of the per-token log-likelihoods of vocab_loss (plain numpy, fp64), written out from
+    Eq. 5: with p[n, v] = exp(Y[n, v] - lse[n]) and an upstream weight dloss[n] per token,
+        dY[n, v] = dloss[n] * ([v == t_n] - p[n, v]),   dX = dY W_voc^T,   dW_voc = X^T dY.
+    declared=True rounds dY to bf16 before the two products (the tensor the CUDA path hands to its
+    tensor-core products in bf16).  Returns (dX [N,H], dW [H,V])."""
+    X = bf16_bits_to_f64(x_bits)
+    W = bf16_bits_to_f64(W_bits)
+    t = np.asarray(targets, np.int64)
+    g = np.asarray(dloss, np.float64)
+    Y = X @ W
+    m = Y.max(1)
+    lse = m + np.log(np.exp(Y - m[:, None]).sum(1))
+    dY = -np.exp(Y - lse[:, None])
+    dY[np.arange(Y.shape[0]), t] += 1.0
+    dY *= g[:, None]
+    if declared:
+        dY = bf16_bits_to_f64(f32_to_bf16_bits(dY.astype(np.float32)))
+    return dY @ W.T, X.T @ dY
+

@@ -426,3 +426,49 @@ def test_vocab_loss_matches_library_cross_entropy_and_closed_forms():
     big = synth.bits((torch.from_numpy(oracle.bf16_bits_to_f32(W)) * 64).to(torch.bfloat16))
     lb, _ = oracle.vocab_loss(x, big, t)
     assert np.all(np.isfinite(lb))
+
+
+def test_vocab_loss_backward_matches_autodiff_finite_differences_and_closed_forms():
+    rng = np.random.default_rng(41)
+    N, H, V = 11, 16, 203
+    x = _rand_bits(rng, (N, H))
+    W = _rand_bits(rng, (H, V), 0.3)
+    t = rng.integers(0, V, N)
+    g = rng.standard_normal(N)
+    dX, dW = oracle.vocab_loss_bwd(x, W, t, g)
+    # (1) library autodiff of the library's own cross entropy (the loss is minus the cross entropy)
+    Xt = torch.tensor(oracle.bf16_bits_to_f64(x), requires_grad=True)
+    Wt = torch.tensor(oracle.bf16_bits_to_f64(W), requires_grad=True)
+    ce = torch.nn.functional.cross_entropy(Xt @ Wt, torch.from_numpy(t), reduction="none")
+    (-(ce * torch.from_numpy(g)).sum()).backward()
+    assert np.max(np.abs(dX - Xt.grad.numpy())) < 1e-11
+    assert np.max(np.abs(dW - Wt.grad.numpy())) < 1e-11
+    # (2) central finite differences of the forward oracle's definition written out here
+    Xf, Wf = oracle.bf16_bits_to_f64(x), oracle.bf16_bits_to_f64(W)
+
+    def total(Xa, Wa):
+        Y = Xa @ Wa
+        m = Y.max(1)
+        lse = m + np.log(np.exp(Y - m[:, None]).sum(1))
+        return float(((Y[np.arange(N), t] - lse) * g).sum())
+
+    eps = 1e-6
+    for (n, h) in ((0, 0), (3, 7), (10, 15)):
+        E = np.zeros_like(Xf); E[n, h] = eps
+        assert abs((total(Xf + E, Wf) - total(Xf - E, Wf)) / (2 * eps) - dX[n, h]) < 1e-6
+    for (h, v) in ((0, int(t[0])), (5, 100), (15, 202)):
+        E = np.zeros_like(Wf); E[h, v] = eps
+        assert abs((total(Xf, Wf + E) - total(Xf, Wf - E)) / (2 * eps) - dW[h, v]) < 1e-6
+    # (3) closed form at W = 0: p is uniform, dY = g ([v == t] - 1/V), so dX = 0 and
+    #     dW[:, v] = sum_n x[n] g[n] ([v == t_n] - 1/V)
+    dX0, dW0 = oracle.vocab_loss_bwd(x, np.zeros_like(W), t, g)
+    assert np.max(np.abs(dX0)) == 0.0
+    onehot = np.zeros((N, V)); onehot[np.arange(N), t] = 1.0
+    assert np.max(np.abs(dW0 - Xf.T @ ((onehot - 1.0 / V) * g[:, None]))) < 1e-12
+    # (4) every row of dY sums to zero: the gradient is orthogonal to a constant shift of a token's logits,
+    #     i.e. dW summed over the vocabulary vanishes
+    assert np.max(np.abs(dW.sum(1))) < 1e-10
+    # (5) the declared-rounding mode differs from the exact one only by the bf16 rounding of dY
+    dXd, dWd = oracle.vocab_loss_bwd(x, W, t, g, declared=True)
+    assert 0 < np.max(np.abs(dXd - dX)) < 2e-2 * max(1.0, np.abs(dX).max())
+    assert np.linalg.norm(dWd - dW) / np.linalg.norm(dW) < 1e-2
