@@ -206,8 +206,10 @@ def run_reference(args, w):
 # --------------------------------------------------------------------------------------- second workload
 def run_vocab(args):
     """Vocabulary projection with online log-likelihood (Eq. 5): N = 8192 tokens, H = 7168, V = 131072
-    (--shape N,H,V overrides).  One step = one forward; the N x V logits are never stored."""
+    (--shape N,H,V overrides).  vocab_loss: one step = one forward; vocab_train: forward + backward
+    (dX, dW_voc).  The N x V logits are never stored."""
     from paper_2607_01844_b200 import binding
+    train = args.workload == "vocab_train"
     N, H, V = (int(v) for v in args.shape.split(",")) if args.shape else (8192, 7168, 131072)
     steps, warmup = args.steps or 10, max(3, args.warmup or 3)
     torch.cuda.set_device(0)
@@ -216,32 +218,50 @@ def run_vocab(args):
     W = (torch.randn((H, V), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
     t = torch.randint(0, V, (N,), generator=g, device="cuda", dtype=torch.int32)
     loss = torch.empty((N,), device="cuda")
-    ws = binding.mop_vocab_loss_fwd(0, X, W, t, loss)
+    lse = torch.empty((N,), device="cuda")
+    ws = binding.mop_vocab_loss_fwd(0, X, W, t, loss, lse)
     stream = torch.cuda.current_stream()
+    ws_b = None
+    if train:
+        dloss = torch.full((N,), -1.0 / N, device="cuda")
+        dX = torch.empty_like(X)
+        dW = torch.empty((H, V), device="cuda")
+        ws_b = binding.mop_vocab_loss_bwd(0, X, W, t, lse, dloss, dX, dW)
+
+    def step():
+        binding.mop_vocab_loss_fwd(0, X, W, t, loss, lse, ws, stream)
+        if train:
+            binding.mop_vocab_loss_bwd(0, X, W, t, lse, dloss, dX, dW, ws_b, stream)
+
     for _ in range(warmup):
-        binding.mop_vocab_loss_fwd(0, X, W, t, loss, None, ws, stream)
+        step()
     sampler = ClockSampler(0)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     sampler.start()
     e0.record(stream)
     for _ in range(steps):
-        binding.mop_vocab_loss_fwd(0, X, W, t, loss, None, ws, stream)
+        step()
     e1.record(stream)
     torch.cuda.synchronize()
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1) / steps
     pk, pk_kind = peaks()
-    tf = 2.0 * N * H * V / (ms * 1e-3) / 1e12
+    blocks = (V + 8191) // 8192
+    # forward: one product; backward: logits again, dW_voc and dX: three more
+    tf = (8.0 if train else 2.0) * N * H * V / (ms * 1e-3) / 1e12
     print(json.dumps({
-        "metric": "vocab_loss_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": steps, "warmup": warmup,
+        "metric": "vocab_train_tflops" if train else "vocab_loss_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": steps, "warmup": warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic", "config": {"workload": "vocab_loss", "N": N, "H": H, "V": V, "l2": "inputs larger than L2"},
-        "clocks": clocks, "gpu_launches": 3 * steps,
-        "roofline": {"kernel": "vocab_logits_lse", "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops_sustained"],
+        "data": "synthetic", "config": {"workload": args.workload, "N": N, "H": H, "V": V, "l2": "inputs larger than L2"},
+        "clocks": clocks, "gpu_launches": (3 + (3 * blocks + 2 if train else 0)) * steps,
+        "roofline": {"kernel": "vocab_logits_lse" + (" + vocab_dlogits + vocab_wgrad + vocab_dgrad" if train else ""),
+                     "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops_sustained"], "peak_source": pk_kind, "traffic": None,
-                     "note": "whole call (tile table + GEMM with online log-sum-exp + merge)"},
-        "logits_never_stored_bytes": N * V * 2, "workspace_bytes": int(ws.numel()),
+                     "note": "whole call(s): tile table + GEMMs with their epilogues + merge / conversion"},
+        "logits_never_stored_bytes": N * V * 2,
+        "workspace_bytes": int(ws.numel()) + (int(ws_b.numel()) if train else 0),
     }))
 
 
@@ -252,7 +272,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c5_train", choices=sorted(synth.WORKLOADS) + ["vocab_loss"])
+    ap.add_argument("--workload", default="c5_train", choices=sorted(synth.WORKLOADS) + ["vocab_loss", "vocab_train"])
     ap.add_argument("--shape", default=None,
                     help="T,d,E,k,f overriding the named workload's sizes (same distributions): small cases for "
                          "profiler captures")
@@ -264,7 +284,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
-    if args.workload == "vocab_loss":
+    if args.workload in ("vocab_loss", "vocab_train"):
         return run_vocab(args)
     w = synth.WORKLOADS[args.workload]
     if args.shape:

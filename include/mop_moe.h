@@ -236,14 +236,30 @@ int32_t mop_profile_read(mop_ctx* ctx, void* stream, int32_t max_names, const ch
  *   Y = X W_voc,   loss[n] = Y[n, t_n] - log sum_v exp(Y[n, v])      (the token's log-likelihood)
  * computed tile by tile on the tensor cores (bf16 operands, fp32 accumulation) with a running
  * maximum and sum per row, so that the N x V logits are never stored: the only intermediate is one
- * (max, sum) pair per row and 256-column block.  One-GPU counterpart of Section 3.4's projection;
- * forward only.  H and V must be multiples of 64.
+ * (max, sum) pair per row and 256-column block.  One-GPU counterpart of Section 3.4's projection.  H and V must be multiples of 64.
  * X [N,H] bf16; W_voc [H,V] bf16; targets [N] i32 in [0,V); loss [N] f32 out; lse_opt [N] f32 out or
  * NULL; workspace: device memory of mop_vocab_workspace_bytes(N, H, V) bytes, 256-byte aligned,
  * owned by the caller (nothing is allocated here).  `device` is the CUDA ordinal. */
 size_t mop_vocab_workspace_bytes(int32_t N, int32_t H, int32_t V);
 mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const void* X, const void* W_voc,
                               const int32_t* targets, float* loss, float* lse_opt, void* workspace, void* stream);
+
+/* Gradients of those log-likelihoods, again without the N x V matrix.  With p[n,v] =
+ * exp(Y[n,v] - lse[n]) and an upstream weight dloss[n] per token (for a mean negative
+ * log-likelihood: -1/N),
+ *   dY[n,v] = dloss[n] ([v == t_n] - p[n,v]),   dX = dY W_voc^T,   dW_voc = X^T dY.
+ * The vocabulary is walked in blocks of 8192 columns: the block's logits are recomputed on the
+ * tensor cores, turned into dY in the epilogue (bf16, N x 8192, the only piece of the N x V matrix
+ * that ever exists), multiplied into dW_voc[:, block] (written once) and accumulated into dX in
+ * fp32 across the blocks (rounded to bf16 at the end).  Eq. 5 defines the loss; its derivative is
+ * written out here.  lse is the output of mop_vocab_loss_fwd.
+ * X [N,H] bf16; W_voc [H,V] bf16; targets [N] i32; lse, dloss [N] f32; dX [N,H] bf16 out;
+ * dW_voc [H,V] f32 out (overwritten); workspace: mop_vocab_bwd_workspace_bytes(N, H, V) bytes of
+ * device memory, 256-byte aligned, owned by the caller. */
+size_t mop_vocab_bwd_workspace_bytes(int32_t N, int32_t H, int32_t V);
+mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const void* X, const void* W_voc,
+                              const int32_t* targets, const float* lse, const float* dloss, void* dX,
+                              float* dW_voc, void* workspace, void* stream);
 
 /* The same permutation as mop_moe_permute for callers that may not allocate device memory (the
  * paper has no counterpart; this is a property of the library, not of the method).  A process

@@ -69,6 +69,9 @@ def lib() -> ctypes.CDLL:
         L.mop_vocab_workspace_bytes.argtypes = [ctypes.c_int32] * 3
         L.mop_vocab_workspace_bytes.restype = ctypes.c_size_t
         L.mop_vocab_loss_fwd.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 3 + [_P] * 7
+        L.mop_vocab_bwd_workspace_bytes.argtypes = [ctypes.c_int32] * 3
+        L.mop_vocab_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.mop_vocab_loss_bwd.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 3 + [_P] * 9
         L.mop_profile_enable.argtypes = [_P, ctypes.c_int]
         L.mop_profile_read.argtypes = [_P, _P, ctypes.c_int32, ctypes.POINTER(ctypes.c_char_p),
                                        ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
@@ -241,6 +244,22 @@ def mop_vocab_loss_fwd(device, X, W_voc, targets, loss, lse=None, workspace=None
     _check("mop_vocab_loss_fwd",
            lib().mop_vocab_loss_fwd(device, N, H, V, _ptr(X), _ptr(W_voc), _ptr(targets), _ptr(loss), _ptr(lse),
                                     _ptr(workspace), _stream(stream)))
+    return workspace
+
+
+def mop_vocab_bwd_workspace_bytes(N, H, V):
+    return lib().mop_vocab_bwd_workspace_bytes(N, H, V)
+
+
+def mop_vocab_loss_bwd(device, X, W_voc, targets, lse, dloss, dX, dW_voc, workspace=None, stream=None):
+    """dX, dW_voc of sum_n dloss[n] * loglik[n]; only an N x 8192 block of the logit gradients is ever live."""
+    N, H = X.shape
+    V = W_voc.shape[1]
+    if workspace is None:
+        workspace = torch.empty(max(256, mop_vocab_bwd_workspace_bytes(N, H, V)), dtype=torch.uint8, device=X.device)
+    _check("mop_vocab_loss_bwd",
+           lib().mop_vocab_loss_bwd(device, N, H, V, _ptr(X), _ptr(W_voc), _ptr(targets), _ptr(lse), _ptr(dloss),
+                                    _ptr(dX), _ptr(dW_voc), _ptr(workspace), _stream(stream)))
     return workspace
 
 

@@ -9,6 +9,8 @@
 //   WD   dW_down[e] = (gate H)_e^T dYp_e          fp32 store                          ragged K
 //   WGU  [dW_gate|dW_up][e] = Xp_e^T [dG|dU]_e    fp32 store                          ragged K
 //   VL   Y = X W_voc (never stored)               online log-sum-exp partials         dense M
+//   VP   dY = g ([v = t] - exp(X W_voc - lse))     bf16, one block of vocabulary columns dense M
+//   VX   dX += dY W_voc^T over that block          fp32 read-modify-write              dense M
 // CTA tile 128 x 256 (one tcgen05.mma.cta_group::1 of M=128, N=256, K=16 per 32 bytes of K),
 // K step 64 per pipeline stage, 4 stages, two 256-column accumulators in TMEM so that the
 // epilogue of tile i overlaps the main loop of tile i+1.
@@ -24,7 +26,7 @@
 
 namespace mop {
 
-enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5, TC_VL = 6 };
+enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5, TC_VL = 6, TC_VP = 7, TC_VX = 8 };
 
 constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // 16 KiB
@@ -37,7 +39,7 @@ constexpr long long TC_WAIT_CYCLES = 4000000000ll;  // about two seconds
 template <int KIND>
 struct TcTraits {
     static constexpr bool A_MN = (KIND == TC_WD || KIND == TC_WGU);   // A is M-contiguous in memory
-    static constexpr bool B_MN = (KIND != TC_B2 && KIND != TC_B4);    // B is N-contiguous in memory
+    static constexpr bool B_MN = (KIND != TC_B2 && KIND != TC_B4 && KIND != TC_VX);   // B is N-contiguous in memory
     static constexpr bool DUAL_B = (KIND == TC_F1 || KIND == TC_WGU); // two B tensors, 128 columns each
     static constexpr bool RAGGED_K = A_MN;
     static constexpr bool B_WEIGHT = !RAGGED_K;                       // B is an [E, ., .] weight tensor
@@ -62,8 +64,12 @@ struct TcArgs {
     int kblocks;             // ragged M: K / 64 (rounded up) per phase
     int Mfix, N;             // ragged K: output rows per expert; N = columns per output tensor
     int m_fastest;           // tile order: 1 = consecutive tiles walk the row tiles of one column block
-    const int32_t* targets;  // VL: target column per row
+    const int32_t* targets;  // VL, VP: target column per row
     float* ylab;             // VL: logit of the target column per row
+    const float* row_lse;    // VP: log-sum-exp per row
+    const float* row_g;      // VP: upstream weight per row
+    int n_base;              // VP: first vocabulary column of the block (added to the tile's columns)
+    int kb_base;             // VX: first vocabulary column of the block (added to B's K coordinate)
     int32_t* status;
     EpiArgs ep;
     float* outf1;            // WGU: second output tensor
@@ -409,6 +415,33 @@ __device__ __forceinline__ void tc_epilogue_rows(const TcArgs& args, uint32_t ta
         if (row_ok) {
             reinterpret_cast<float2*>(args.ep.part)[(size_t)nt * args.ep.M_total + grow] = make_float2(m, ssum);
         }
+    } else if constexpr (KIND == TC_VP) {
+        // Gradient of the log-likelihood with respect to the logits of this block of the vocabulary,
+        // from the recomputed logits and the row's log-sum-exp; bf16, block-local columns.
+        const float lse = row_ok ? args.row_lse[grow] : 0.0f;
+        const float g = row_ok ? args.row_g[grow] : 0.0f;
+        const int tgt = row_ok ? args.targets[grow] - n0 : -1;
+#pragma unroll 1
+        for (int c = 0; c < TC_BN; c += 32) {
+            tmem_ld32(taddr + c, acc);
+            if (row_ok && n0 + c < args.N) {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) acc[q] = g * ((tgt - c == q ? 1.0f : 0.0f) - __expf(acc[q] - lse));
+#pragma unroll
+                for (int s = 0; s < 32; s += 8) {
+                    float a8[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) a8[q] = acc[s + q];
+                    store_bf16_run<8>(args.ep.out0 + (size_t)grow * args.ep.ldo + (n0 - args.n_base) + c + s, a8);
+                }
+            }
+        }
+    } else if constexpr (KIND == TC_VX) {
+#pragma unroll 1
+        for (int c = 0; c < TC_BN; c += 32) {
+            tmem_ld32(taddr + c, acc);
+            if (row_ok && n0 + c < args.N) epi_f32<32>(args.ep.outf + (size_t)grow * args.N + n0 + c, acc, args.ep.accumulate);
+        }
     } else if constexpr (KIND == TC_B4) {
 #pragma unroll 1
         for (int c = 0; c < TC_BN; c += 32) {
@@ -482,7 +515,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 const TileInfo ti = nxt;
                 if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
                 if (ti.skip) continue;
-                const int n0 = ti.nt * Tr::N_PER_TILE;
+                const int n0 = ti.nt * Tr::N_PER_TILE + (KIND == TC_VP ? args.n_base : 0);
                 const int nkb = Tr::RAGGED_K ? (ti.rows + TC_BK - 1) / TC_BK : Tr::PHASES * args.kblocks;
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) {
@@ -501,7 +534,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                         tma_load_3d_hint(sA, &tmA0, fb, 0, ti.row0 + kb * TC_BK, ti.m0 >> 6, keep);
                     }
                     if constexpr (!Tr::B_MN) {
-                        tma_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0, n0, ti.e);
+                        tma_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0 + (KIND == TC_VX ? args.kb_base : 0), n0, ti.e);
                     } else {
                         // chunked maps {64, rows, cols/64 [, E]}: the 64-wide column chunks of the tile arrive
                         // chunk-major in one copy per tensor (four chunks, or two each of two tensors)
@@ -589,7 +622,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             const TileInfo ti = nxt;
             if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
-            const int n0 = ti.nt * Tr::N_PER_TILE;
+            const int n0 = ti.nt * Tr::N_PER_TILE + (KIND == TC_VP ? args.n_base : 0);
             if constexpr (Tr::RAGGED_K) {
                 if (ti.skip) {
                     // expert without rows: its gradient is zero (or unchanged when accumulating)
@@ -702,6 +735,15 @@ __global__ void vocab_lse_merge_kernel(const float2* __restrict__ part, const fl
     loss[n] = ylab[n] - l;
 }
 
+// fp32 -> bf16 of a dense array (8 elements per thread; n a multiple of 8)
+__global__ void f32_to_bf16_kernel(const float4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+        const float4 a = src[2 * i], b = src[2 * i + 1];
+        const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        store_bf16_run<8>(reinterpret_cast<bf16*>(dst + i), v);
+    }
+}
+
 // ------------------------------------------------------------------------------------------ host
 struct TcPlan {
     int sm_count;
@@ -758,6 +800,8 @@ inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count, 
     if ((r = tc_set_smem<TC_WD>()) != MOP_OK) return r;
     if ((r = tc_set_smem<TC_WGU>()) != MOP_OK) return r;
     if ((r = tc_set_smem<TC_VL>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_VP>()) != MOP_OK) return r;
+    if ((r = tc_set_smem<TC_VX>()) != MOP_OK) return r;
     return MOP_OK;
 }
 
@@ -810,6 +854,42 @@ inline bool tc_map_chunked_3d(const TcPlan* p, CUtensorMap* m, const void* base,
     return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base),
                                                      dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same views over a column block of a wider matrix: `cols` columns starting at `base`, rows
+// `pitch` elements apart (pitch * element size and base must be multiples of 16 bytes).
+inline bool tc_map_2d_pitch(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                            uint64_t pitch, uint32_t box_rows) {
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t es[2] = {1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+inline bool tc_map_chunked_2d_pitch(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                                    uint64_t pitch, uint32_t chunks) {
+    const cuuint64_t dims[3] = {64, rows, cols / 64};
+    const cuuint64_t strides[2] = {pitch * 2, 128};
+    const cuuint32_t box[3] = {64, 64, chunks};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+inline bool tc_map_out_f32_pitch(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                                 uint64_t pitch) {
+    const cuuint64_t dims[3] = {cols, rows, 1};
+    const cuuint64_t strides[2] = {pitch * 4, rows * pitch * 4};
+    const cuuint32_t box[3] = {32, 128, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base),
+                                                     dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -1058,4 +1058,113 @@ mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
+namespace {
+constexpr int kVocabBlock = 8192;   // vocabulary columns whose logit gradients are live at a time
+struct VocabBwdLayout { size_t off, tiles, status, dy, dx32, total; int vc; };
+VocabBwdLayout vocab_bwd_layout(int N, int H, int V) {
+    VocabBwdLayout L{};
+    size_t o = 0;
+    auto take = [&](size_t b) { size_t r = o; o += align_up(b); return r; };
+    L.vc = V < kVocabBlock ? V : kVocabBlock;
+    L.off = take(16);
+    L.tiles = take(tc_tile_table_bytes(N, 1));
+    L.status = take(256);
+    L.dy = take((size_t)N * L.vc * 2);
+    L.dx32 = take((size_t)N * H * 4);
+    L.total = o;
+    return L;
+}
+mop_status vocab_plan(int device, TcPlan** out) {
+    TcPlan* p = &g_vocab_plan[device];
+    std::lock_guard<std::mutex> lock(g_vocab_mutex);
+    if (!g_vocab_ready[device]) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MOP_ERR_CUDA;
+        if (prop.major != 10) return MOP_ERR_UNSUPPORTED;
+        mop_moe_shape dummy{};
+        mop_status r = tc_plan_init(p, dummy, prop.multiProcessorCount, &g_vocab_prof);
+        if (r != MOP_OK) return r;
+        g_vocab_ready[device] = true;
+    }
+    *out = p;
+    return MOP_OK;
+}
+}  // namespace
+
+size_t mop_vocab_bwd_workspace_bytes(int32_t N, int32_t H, int32_t V) {
+    if (N < 0 || H < 64 || V < 64 || H % 64 || V % 64) return 0;
+    return vocab_bwd_layout(N, H, V).total;
+}
+
+mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const void* X, const void* W_voc,
+                              const int32_t* targets, const float* lse, const float* dloss, void* dX, float* dW_voc,
+                              void* workspace, void* stream) {
+    if (N < 0 || H < 1 || V < 1) return MOP_ERR_INVALID_ARG;
+    if (H % 64 || V % 64) return MOP_ERR_UNSUPPORTED;
+    if ((long long)N * 2 >= (1ll << 31) || (long long)H * V >= (1ll << 40)) return MOP_ERR_SHAPE;
+    if (!W_voc || !dW_voc || !workspace) return MOP_ERR_INVALID_ARG;
+    if (N > 0 && (!X || !targets || !lse || !dloss || !dX)) return MOP_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(W_voc) || !aligned16(targets) || !aligned16(lse) || !aligned16(dloss) ||
+        !aligned16(dX) || !aligned16(dW_voc) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return MOP_ERR_ALIGN;
+    if (device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (N == 0) {   // no tokens: the weight gradient is zero
+        CUDA_OK(cudaMemsetAsync(dW_voc, 0, (size_t)H * V * 4, st));
+        return MOP_OK;
+    }
+    TcPlan* p = nullptr;
+    mop_status r = vocab_plan(device, &p);
+    if (r != MOP_OK) return r;
+    const VocabBwdLayout L = vocab_bwd_layout(N, H, V);
+    char* w = static_cast<char*>(workspace);
+    int32_t* off = reinterpret_cast<int32_t*>(w + L.off);
+    int32_t* tiles = reinterpret_cast<int32_t*>(w + L.tiles);
+    int32_t* status = reinterpret_cast<int32_t*>(w + L.status);
+    bf16* dY = reinterpret_cast<bf16*>(w + L.dy);
+    float* dx32 = reinterpret_cast<float*>(w + L.dx32);
+    const int32_t host_off[2] = {0, N};
+    CUDA_OK(cudaMemcpyAsync(off, host_off, sizeof(host_off), cudaMemcpyHostToDevice, st));
+    CUDA_OK(cudaMemsetAsync(status, 0, 4, st));
+    tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
+    CUtensorMap mX, mXT, mWn, mWk;
+    if (!tc_map_2d(p, &mX, X, N, H, 128) || !tc_map_chunked_2d(p, &mXT, X, N, H, 2) ||
+        !tc_map_chunked_3d(p, &mWn, W_voc, 1, H, V, 4) || !tc_map_3d(p, &mWk, W_voc, 1, H, V, 256))
+        return MOP_ERR_CUDA;
+    for (int c0 = 0; c0 < V; c0 += L.vc) {
+        const int cw = V - c0 < L.vc ? V - c0 : L.vc;
+        CUtensorMap mdYk, mdYn, mOut;
+        if (!tc_map_2d_pitch(p, &mdYk, dY, N, cw, L.vc, 128) || !tc_map_chunked_2d_pitch(p, &mdYn, dY, N, cw, L.vc, 4) ||
+            !tc_map_out_f32_pitch(p, &mOut, dW_voc + c0, H, cw, V))
+            return MOP_ERR_CUDA;
+        TcArgs base{};
+        base.offsets = off; base.n_mtiles = tiles; base.mtiles = reinterpret_cast<const int4*>(tiles + 64);
+        base.E = 1; base.status = status; base.ep.M_total = N;
+        {   // dY block = g ([v = t] - exp(X W - lse)), logits recomputed on the tensor cores
+            TcArgs g = base;
+            g.tiles_n = ceil_div(cw, 256); g.kblocks = ceil_div(H, TC_BK); g.N = V; g.m_fastest = 1; g.n_base = c0;
+            g.targets = targets; g.row_lse = lse; g.row_g = dloss; g.ep.out0 = dY; g.ep.ldo = L.vc;
+            if ((r = tc_launch<TC_VP>(p, "vocab_dlogits", mX, mX, mWn, mWn, mX, mX, g, st)) != MOP_OK) return r;
+        }
+        {   // dW[:, block] = X^T dY (K = the N tokens), written once
+            TcArgs g = base;
+            g.tiles_n = ceil_div(cw, 256); g.tiles_m_fixed = ceil_div(H, TC_BM); g.Mfix = H; g.N = cw;
+            g.ep.outf = dW_voc + c0; g.ep.accumulate = 0;
+            if ((r = tc_launch<TC_WD>(p, "vocab_wgrad", mXT, mXT, mdYn, mdYn, mOut, mOut, g, st)) != MOP_OK) return r;
+        }
+        {   // dX += dY W[:, block]^T in fp32 across the blocks
+            TcArgs g = base;
+            g.tiles_n = ceil_div(H, 256); g.kblocks = ceil_div(cw, TC_BK); g.N = H; g.kb_base = c0;
+            g.ep.outf = dx32; g.ep.accumulate = c0 > 0 ? 1 : 0;
+            if ((r = tc_launch<TC_VX>(p, "vocab_dgrad", mdYk, mdYk, mWk, mWk, mX, mX, g, st)) != MOP_OK) return r;
+        }
+    }
+    const size_t n8 = (size_t)N * H / 8;
+    f32_to_bf16_kernel<<<(unsigned)((n8 + 255) / 256 < 148 * 16 ? (n8 + 255) / 256 : 148 * 16), 256, 0, st>>>(
+        reinterpret_cast<const float4*>(dx32), static_cast<uint4*>(dX), n8);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
+
 }  // extern "C"

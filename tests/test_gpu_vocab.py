@@ -57,3 +57,72 @@ def test_vocab_loss_rejects_bad_arguments():
         binding.mop_vocab_loss_fwd(0, X[:, :32].contiguous(), W[:32].contiguous(), t, loss)     # H = 32
     assert e.value.code == 6
     assert binding.mop_vocab_workspace_bytes(64, 64, 100) == 0
+
+
+def _rel_fro(got, ref):
+    n = np.linalg.norm(ref)
+    return float(np.linalg.norm(got - ref) / (n if n > 0 else 1.0))
+
+
+@pytest.mark.parametrize("N,H,V,std", [(1, 64, 64, 0.3), (300, 128, 1024, 0.2), (200, 128, 8192 + 320, 0.1),
+                                       (513, 256, 16384 + 64, 0.05), (129, 192, 320, 1.0)])
+def test_vocab_loss_backward_matches_oracle(N, H, V, std):
+    """dX and dW_voc against the fp64 oracle; the shapes span one, two and three vocabulary blocks with ragged tails."""
+    X, W, t = _inputs(N, H, V, seed=N + V + 1, std=std)
+    t[0] = 0
+    t[-1] = V - 1
+    g = torch.randn((N,), device="cuda") * 0.5 - 1.0
+    loss = torch.empty((N,), device="cuda")
+    lse = torch.empty((N,), device="cuda")
+    binding.mop_vocab_loss_fwd(0, X, W, t, loss, lse)
+    dX = torch.full((N, H), 3.0, device="cuda", dtype=torch.bfloat16)
+    dW = torch.full((H, V), 3.0, device="cuda")
+    binding.mop_vocab_loss_bwd(0, X, W, t, lse, g, dX, dW)
+    torch.cuda.synchronize()
+    xb, wb, tn, gn = synth.bits(X), synth.bits(W), t.cpu().numpy(), g.cpu().numpy()
+    dX_e, dW_e = oracle.vocab_loss_bwd(xb, wb, tn, gn)
+    dX_d, dW_d = oracle.vocab_loss_bwd(xb, wb, tn, gn, declared=True)
+    gX, gW = dX.float().cpu().numpy().astype(np.float64), dW.cpu().numpy().astype(np.float64)
+    assert _rel_fro(gX, dX_e) <= 1e-2 and _rel_fro(gW, dW_e) <= 1e-2
+    # against the declared-rounding mode only summation order, __expf and the final bf16 of dX remain
+    assert np.max(np.abs(gX - dX_d)) <= 2e-2 * max(1.0, float(np.abs(dX_d).max()))
+    assert np.max(np.abs(gW - dW_d)) <= 2e-2 * max(1.0, float(np.abs(dW_d).max()))
+    # reproducible bit for bit
+    dX2, dW2 = torch.empty_like(dX), torch.empty_like(dW)
+    binding.mop_vocab_loss_bwd(0, X, W, t, lse, g, dX2, dW2)
+    assert torch.equal(dX, dX2) and torch.equal(dW, dW2)
+
+
+def test_vocab_loss_backward_without_tokens_zeroes_the_weight_gradient():
+    X, W, t = _inputs(0, 64, 128, seed=3)
+    dW = torch.full((64, 128), 3.0, device="cuda")
+    dX = torch.empty((0, 64), device="cuda", dtype=torch.bfloat16)
+    e = torch.empty((0,), device="cuda")
+    ws = torch.empty(max(256, binding.mop_vocab_bwd_workspace_bytes(0, 64, 128)), dtype=torch.uint8, device="cuda")
+    binding.mop_vocab_loss_bwd(0, X, W, t, e, e, dX, dW, ws)
+    torch.cuda.synchronize()
+    assert float(dW.abs().max()) == 0.0
+
+
+def test_vocab_loss_backward_full_size_sampled_rows_and_invariant():
+    """N = 8192, H = 7168, V = 131072 (sixteen vocabulary blocks): dX of sampled tokens against the oracle,
+    and the vocabulary sum of dW_voc, which vanishes because every row of dY sums to zero."""
+    N, H, V = 8192, 7168, 131072
+    X, W, t = _inputs(N, H, V, seed=6)
+    loss = torch.empty((N,), device="cuda")
+    lse = torch.empty((N,), device="cuda")
+    binding.mop_vocab_loss_fwd(0, X, W, t, loss, lse)
+    g = torch.full((N,), -1.0, device="cuda")
+    dX = torch.empty_like(X)
+    dW = torch.empty((H, V), device="cuda")
+    binding.mop_vocab_loss_bwd(0, X, W, t, lse, g, dX, dW)
+    torch.cuda.synchronize()
+    rows = np.sort(np.random.default_rng(6).choice(N, 4, replace=False))
+    r = torch.as_tensor(rows, device="cuda")
+    dX_e, _ = oracle.vocab_loss_bwd(synth.bits(X[r]), synth.bits(W), t[r].cpu().numpy(), g[r].cpu().numpy())
+    got = dX[r].float().cpu().numpy().astype(np.float64)
+    assert _rel_fro(got, dX_e) <= 1e-2
+    col_sum = dW.sum(1, dtype=torch.float64)
+    scale = dW.abs().sum(1, dtype=torch.float64)
+    assert float((col_sum.abs() / scale).max()) < 2e-3      # bf16 rounding of dY leaves a small residue
+    assert torch.isfinite(dW).all()
