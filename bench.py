@@ -388,7 +388,7 @@ def main():
         for _ in range(2):
             host_step()
         binding.mop_host_drain(ctx, stream)
-        n_e2e = min(args.steps, 10)
+        n_e2e = args.steps
         barrier(); torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
