@@ -249,44 +249,43 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         }
     } else if (warp == 1) {
         // ===================================================================== MMA issuer (leader CTA)
-        if (leader) {
+        // One thread runs the whole loop (wait, fence, four MMAs, commit): per K block nothing but
+        // these instructions stands between two groups of MMAs, so the tensor pipe's queue stays fed.
+        if (leader && lane == 0) {
+            constexpr bool A_KMAJOR = (KIND == TN_B4 || KIND == TN_B2);
+            // descriptors without the start address: A is M-major (N-major weights) or K-major, B is K-major
+            const uint64_t desc_a = smem_desc(0, A_KMAJOR ? 0 : TC_CHUNK_BYTES, 1024);
+            const uint64_t desc_b = smem_desc(0, 0, 1024);
+            constexpr uint32_t a_step = (A_KMAJOR ? 32 : 2048) >> 4;    // start-address field advance per K = 16
             int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
             Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
                 const Tile ti = nxt;
                 if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
-                // A is M-major (N-major weights; K-major for B4), B is K-major; M = 256 over the pair,
-                // N = this tile's tokens
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((KIND == TN_B4 || KIND == TN_B2 ? 0u : 1u) << 15) |
+                // M = 256 over the pair, N = this tile's tokens
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_KMAJOR ? 0u : 1u) << 15) |
                                        ((uint32_t)(ti.nmma >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
                 const int buf = it & 1;
                 const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait_warp(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY, lane))
-                    break;
+                if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * 256;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait_warp(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL, lane)) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL)) {
                         alive = false; break;
                     }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
-                    const uint32_t sB = sA + TN_A_BYTES;
-                    if (lane == 0) {
+                    const uint64_t da = desc_a | (uint64_t)((sA & 0x3ffffu) >> 4);
+                    const uint64_t db = desc_b | (uint64_t)(((sA + TN_A_BYTES) & 0x3ffffu) >> 4);
 #pragma unroll
-                        for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
-                            const uint64_t da = (KIND == TN_B4 || KIND == TN_B2) ? smem_desc(sA + k4 * 32, 0, 1024)
-                                                                : smem_desc(sA + k4 * 2048, TC_CHUNK_BYTES, 1024);
-                            umma2_bf16(d_tmem, da, smem_desc(sB + k4 * 32, 0, 1024), idesc, (kb | k4) != 0 ? 1u : 0u);
-                        }
-                        umma2_commit_both(empty_bar(stage));
-                    }
-                    __syncwarp();
+                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
+                        umma2_bf16(d_tmem, da + k4 * a_step, db + k4 * 2, idesc, (kb | k4) != 0 ? 1u : 0u);
+                    umma2_commit_both(empty_bar(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 if (!alive) break;
-                if (lane == 0) umma2_commit_both(tfull_bar(buf));
-                __syncwarp();
+                umma2_commit_both(tfull_bar(buf));
                 ++it;
             }
         }
