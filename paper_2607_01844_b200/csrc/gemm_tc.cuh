@@ -559,6 +559,41 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         constexpr uint32_t mn_lbo = TC_CHUNK_BYTES, mn_sbo = 1024u;
         int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
         TileInfo nxt = decode_tile<KIND>(args, min((int)blockIdx.x, max(total_tiles - 1, 0)));
+        if constexpr (!Tr::RAGGED_K) {
+            // Token-row kinds: one thread runs the whole issue loop (wait, fence, four MMAs, commit) with
+            // descriptors that only need the stage's start address added, so the tensor pipe's queue stays fed.
+            if (lane == 0) {
+                const uint64_t desc_a = smem_desc(0, 0, 1024);
+                const uint64_t desc_b = Tr::B_MN ? smem_desc(0, mn_lbo, mn_sbo) : smem_desc(0, 0, 1024);
+                constexpr uint32_t b_step = (Tr::B_MN ? 2048 : 32) >> 4;
+                const int nkb = Tr::PHASES * args.kblocks;
+                for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+                    if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
+                    const int buf = it & 1;
+                    const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
+                    if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY)) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)buf * TC_BN;
+                    for (int kb = 0; kb < nkb; ++kb) {
+                        if (!mbar_wait(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL)) {
+                            alive = false; break;
+                        }
+                        tc_fence_after();
+                        const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
+                        const uint64_t da = desc_a | (uint64_t)((sA & 0x3ffffu) >> 4);
+                        const uint64_t db = desc_b | (uint64_t)(((sA + TC_A_BYTES) & 0x3ffffu) >> 4);
+#pragma unroll
+                        for (int k4 = 0; k4 < TC_BK / 16; ++k4)
+                            umma_bf16(d_tmem, da + k4 * 2, db + k4 * b_step, idesc, (kb | k4) != 0 ? 1u : 0u);
+                        umma_commit(empty_bar(stage));
+                        if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!alive) break;
+                    umma_commit(tfull_bar(buf));
+                    ++it;
+                }
+            }
+        } else
         for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
             const TileInfo ti = nxt;
             if (t + (int)gridDim.x < total_tiles) nxt = decode_tile<KIND>(args, t + gridDim.x);
