@@ -881,10 +881,10 @@ inline bool tc_map_chunked_2d(const TcPlan* p, CUtensorMap* m, const void* base,
                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 inline bool tc_map_chunked_3d(const TcPlan* p, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows,
-                              uint64_t cols, uint32_t chunks) {
+                              uint64_t cols, uint32_t chunks, uint32_t box_rows = 64) {
     const cuuint64_t dims[4] = {64, rows, cols / 64, E};
     const cuuint64_t strides[3] = {cols * 2, 128, rows * cols * 2};
-    const cuuint32_t box[4] = {64, 64, chunks, 1};
+    const cuuint32_t box[4] = {64, box_rows, chunks, 1};
     const cuuint32_t es[4] = {1, 1, 1, 1};
     return reinterpret_cast<tc_encode_fn>(p->encode)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base),
                                                      dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,

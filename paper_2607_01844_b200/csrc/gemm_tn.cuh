@@ -32,9 +32,11 @@ namespace mop {
 
 enum : int { TN_F1 = 0, TN_F2 = 1, TN_F1G = 2, TN_B4 = 3, TN_B2 = 4 };
 
-constexpr int TN_STAGES = 5;
-constexpr int TN_A_BYTES = 128 * TC_BK * 2;          // 16 KiB: this CTA's 128 weight rows
-constexpr int TN_B_BYTES = 128 * TC_BK * 2;          // up to 128 token rows (half of N = 256)
+constexpr int TN_STAGES = 3;
+constexpr int TN_BK = 128;                           // K per pipeline stage: two 64-wide swizzle spans
+constexpr int TN_SUB_BYTES = 128 * 64 * 2;           // 16 KiB: 128 rows x 64 K (or one 64-wide MN chunk x 128 K)
+constexpr int TN_A_BYTES = 2 * TN_SUB_BYTES;         // 32 KiB: this CTA's 128 weight rows x 128 K
+constexpr int TN_B_BYTES = 2 * TN_SUB_BYTES;         // up to 128 token rows (half of N = 256) x 128 K
 constexpr int TN_STAGE_BYTES = TN_A_BYTES + TN_B_BYTES;
 constexpr int TN_EPI_BYTES = 4 * 8192;               // per epilogue warp: transposition buffers
 constexpr int TN_SMEM_BYTES = TN_STAGES * TN_STAGE_BYTES + 1024 /*align*/ + TC_BAR_BYTES + TN_EPI_BYTES;
@@ -45,7 +47,7 @@ struct TnArgs {
     const int4* ttiles;       // {expert, first row, rows (1..256), 0} per token tile
     const int32_t* n_ttiles;  // device scalar
     int tiles_m;              // weight-row tiles per token tile (each 256 rows; F1: 128 columns of f)
-    int kblocks;              // K / 64 rounded up
+    int kblocks;              // K / 128 rounded up
     int Mw;                   // weight rows in total (F1: f; F2: d)
     const int32_t* row_src;   // F1G: assignment index t*k + j of every expert-contiguous row
     int topk;                 // F1G: k (token of a row = row_src / k)
@@ -180,7 +182,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
                 for (int j = 0; j < 4; ++j) tok[j] = __ldg(args.row_src + min(brow0 + 4 * lane + j, last)) / args.topk;
             }
-            const uint32_t tx = 2u * (TN_A_BYTES + (uint32_t)half * 128u);
+            const uint32_t tx = 2u * (TN_A_BYTES + 2u * (uint32_t)half * 128u);
             for (int kb = 0; kb < args.kblocks; ++kb) {
                 if (!mbar_wait_warp(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY, lane)) {
                     alive = false; break;
@@ -188,14 +190,17 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                 const uint32_t fb = full_bar(stage) & T2_PEER_MASK;
                 const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
                 const uint32_t sB = sA + TN_A_BYTES;
-                const int k0 = kb * TC_BK;
+                const int k0 = kb * TN_BK;
                 if (lane == 0) {
                     if (leader) mbar_expect_tx(full_bar(stage), tx);
                     const int f0 = ti.mt * 128 + 64 * (int)rank;
                     tma2_load_4d(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e);
-                    tma2_load_4d(sA + TC_CHUNK_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e);
+                    tma2_load_4d(sA + TN_SUB_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e);
                 }
-                if (lane < ngroups) tma2_gather4(sB + lane * 512, &tmB, fb, k0, tok[0], tok[1], tok[2], tok[3]);
+                if (lane < ngroups) {
+                    tma2_gather4(sB + lane * 512, &tmB, fb, k0, tok[0], tok[1], tok[2], tok[3]);
+                    tma2_gather4(sB + TN_SUB_BYTES + lane * 512, &tmB, fb, k0 + 64, tok[0], tok[1], tok[2], tok[3]);
+                }
                 __syncwarp();
                 if (++stage == S) { stage = 0; phase ^= 1u; }
             }
@@ -212,7 +217,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                 const int half = ti.nmma >> 1;                         // token rows per CTA
                 const int nbox = (half + TN_BOX_ROWS - 1) / TN_BOX_ROWS;
                 const int brow0 = ti.row0 + (int)rank * half;
-                const uint32_t tx = 2u * (TN_A_BYTES + (uint32_t)nbox * TN_BOX_ROWS * 128u);
+                const uint32_t tx = 2u * (TN_A_BYTES + 2u * (uint32_t)nbox * TN_BOX_ROWS * 128u);
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) {
                         alive = false; break;
@@ -222,13 +227,14 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     const uint32_t sA = smem_base + stage * TN_STAGE_BYTES;
                     const uint32_t sB = sA + TN_A_BYTES;
                     const int ph = (KIND == TN_B4 && kb >= args.kblocks) ? 1 : 0;   // B4: gate phase, then up phase
-                    const int k0 = (kb - ph * args.kblocks) * TC_BK;
+                    const int k0 = (kb - ph * args.kblocks) * TN_BK;
                     if constexpr (KIND == TN_B4 || KIND == TN_B2) {
-                        // K-major weights: this CTA's 128 weight rows, 64 columns of K, one box
+                        // K-major weights: this CTA's 128 weight rows, two boxes of 64 columns of K
                         const int m0 = ti.mt * 256 + 128 * (int)rank;
                         tma2_load_3d(sA, ph ? &tmA1 : &tmA0, fb, k0, m0, ti.e);
-                        for (int b = 0; b < nbox; ++b)
-                            tma2_load_2d(sB + b * TN_BOX_ROWS * 128, ph ? &tmB1 : &tmB, fb, k0, brow0 + b * TN_BOX_ROWS);
+                        tma2_load_3d(sA + TN_SUB_BYTES, ph ? &tmA1 : &tmA0, fb, k0 + 64, m0, ti.e);
+                        tma2_load_2d(sB, ph ? &tmB1 : &tmB, fb, k0, brow0);
+                        tma2_load_2d(sB + TN_SUB_BYTES, ph ? &tmB1 : &tmB, fb, k0 + 64, brow0);
                         if (++stage == S) { stage = 0; phase ^= 1u; }
                         continue;
                     }
@@ -236,13 +242,13 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                         // 64 gate columns, then the 64 matching up columns (N-major weights [E, d, f])
                         const int f0 = ti.mt * 128 + 64 * (int)rank;
                         tma2_load_4d_hint(sA, &tmA0, fb, 0, k0, f0 >> 6, ti.e, pol_w);
-                        tma2_load_4d_hint(sA + TC_CHUNK_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e, pol_w);
+                        tma2_load_4d_hint(sA + TN_SUB_BYTES, &tmA1, fb, 0, k0, f0 >> 6, ti.e, pol_w);
                     } else {
                         const int m0 = ti.mt * 256 + 128 * (int)rank;
                         tma2_load_4d_hint(sA, &tmA0, fb, 0, k0, m0 >> 6, ti.e, pol_w);   // two chunks in one copy
                     }
-                    for (int b = 0; b < nbox; ++b)
-                        tma2_load_2d(sB + b * TN_BOX_ROWS * 128, &tmB, fb, k0, brow0 + b * TN_BOX_ROWS);
+                    tma2_load_2d(sB, &tmB, fb, k0, brow0);
+                    tma2_load_2d(sB + TN_SUB_BYTES, &tmB, fb, k0 + 64, brow0);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -254,9 +260,10 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (leader && lane == 0) {
             constexpr bool A_KMAJOR = (KIND == TN_B4 || KIND == TN_B2);
             // descriptors without the start address: A is M-major (N-major weights) or K-major, B is K-major
-            const uint64_t desc_a = smem_desc(0, A_KMAJOR ? 0 : TC_CHUNK_BYTES, 1024);
+            // A M-major: the two 64-wide chunks are TN_SUB_BYTES apart and hold 128 K rows each (2 KiB per
+            // K = 16); K-major operands: two 64-K sub-tiles TN_SUB_BYTES apart, 32 bytes per K = 16 inside one
+            const uint64_t desc_a = smem_desc(0, A_KMAJOR ? 0 : TN_SUB_BYTES, 1024);
             const uint64_t desc_b = smem_desc(0, 0, 1024);
-            constexpr uint32_t a_step = (A_KMAJOR ? 32 : 2048) >> 4;    // start-address field advance per K = 16
             int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
             Tile nxt = decode(min(cluster_id, max(total_tiles - 1, 0)));
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
@@ -279,8 +286,11 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                     const uint64_t da = desc_a | (uint64_t)((sA & 0x3ffffu) >> 4);
                     const uint64_t db = desc_b | (uint64_t)(((sA + TN_A_BYTES) & 0x3ffffu) >> 4);
 #pragma unroll
-                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
-                        umma2_bf16(d_tmem, da + k4 * a_step, db + k4 * 2, idesc, (kb | k4) != 0 ? 1u : 0u);
+                    for (int k8 = 0; k8 < TN_BK / 16; ++k8) {
+                        const uint32_t kmaj = (uint32_t)((k8 >> 2) * (TN_SUB_BYTES >> 4) + (k8 & 3) * 2);
+                        umma2_bf16(d_tmem, da + (A_KMAJOR ? kmaj : (uint32_t)(k8 * (2048 >> 4))), db + kmaj, idesc,
+                                   (kb | k8) != 0 ? 1u : 0u);
+                    }
                     umma2_commit_both(empty_bar(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -463,11 +473,11 @@ inline mop_status tn_up_swiglu(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, in
     const mop_moe_shape& s = p->s;
     const uint64_t M = (uint64_t)s.T * s.k;
     CUtensorMap mXp, mWg, mWu;
-    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1) ||
-        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1))
+    if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1, 128) ||
+        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1, 128))
         return MOP_ERR_CUDA;
     TnArgs g = tn_base_args(tiles, status);
-    g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
+    g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TN_BK); g.Mw = s.f;
     g.ep.out0 = a.H; g.ep.out1 = a.G_save; g.ep.out2 = a.U_save; g.ep.ldo = s.f; g.ep.M_total = (int)M;
     p->prof->begin("gemm_up_swiglu", st);
     tn_gemm_kernel<TN_F1><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mXp, mXp, g);
@@ -480,11 +490,11 @@ inline mop_status tn_up_swiglu_gather(TcPlan* p, const bf16* x, const TcFwdArgs&
                                       cudaStream_t st) {
     const mop_moe_shape& s = p->s;
     CUtensorMap mX, mWg, mWu;
-    if (!tc_map_2d(p, &mX, x, s.T, s.d, 1) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1) ||
-        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1))
+    if (!tc_map_2d(p, &mX, x, s.T, s.d, 1) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1, 128) ||
+        !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1, 128))
         return MOP_ERR_CUDA;
     TnArgs g = tn_base_args(tiles, status);
-    g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
+    g.tiles_m = ceil_div(s.f, 128); g.kblocks = ceil_div(s.d, TN_BK); g.Mw = s.f;
     g.row_src = a.row_src; g.topk = s.k;
     g.ep.out0 = a.H; g.ep.ldo = s.f; g.ep.M_total = s.T * s.k;
     p->prof->begin("gemm_up_swiglu_gather", st);
@@ -498,10 +508,10 @@ inline mop_status tn_down_gate(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, in
     const mop_moe_shape& s = p->s;
     const uint64_t M = (uint64_t)s.T * s.k;
     CUtensorMap mH, mWd;
-    if (!tc_map_2d(p, &mH, a.H, M, s.f, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 2))
+    if (!tc_map_2d(p, &mH, a.H, M, s.f, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 2, 128))
         return MOP_ERR_CUDA;
     TnArgs g = tn_base_args(tiles, status);
-    g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.Mw = s.d;
+    g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TN_BK); g.Mw = s.d;
     g.ep.out0 = a.Yp; g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.ldo = s.d; g.ep.M_total = (int)M;
     p->prof->begin("gemm_down_gate", st);
     tn_gemm_kernel<TN_F2><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWd, mWd, mH, mH, g);
@@ -518,7 +528,7 @@ inline mop_status tn_dgrad_gate_up(TcPlan* p, const TcBwdArgs& a, int32_t* tiles
         !tc_map_2d(p, &mdG, a.dG, M, s.f, TN_BOX_ROWS) || !tc_map_2d(p, &mdU, a.dU, M, s.f, TN_BOX_ROWS))
         return MOP_ERR_CUDA;
     TnArgs g = tn_base_args(tiles, status);
-    g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TC_BK); g.Mw = s.d;
+    g.tiles_m = ceil_div(s.d, 256); g.kblocks = ceil_div(s.f, TN_BK); g.Mw = s.d;
     g.ep.out0 = a.dXp; g.ep.ldo = s.d; g.ep.M_total = (int)M;
     p->prof->begin("gemm_dgrad_gate_up", st);
     tn_gemm_kernel<TN_B4><<<p->sm_count & ~1, TN_THREADS, TN_SMEM_BYTES, st>>>(mWg, mWu, mdG, mdU, g);
@@ -535,7 +545,7 @@ inline mop_status tn_dgrad_down(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, i
     if (!tc_map_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 128) || !tc_map_2d(p, &mdYp, a.dYp, M, s.d, TN_BOX_ROWS))
         return MOP_ERR_CUDA;
     TnArgs g = tn_base_args(tiles, status);
-    g.tiles_m = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TC_BK); g.Mw = s.f;
+    g.tiles_m = ceil_div(s.f, 256); g.kblocks = ceil_div(s.d, TN_BK); g.Mw = s.f;
     g.ep.out0 = a.dG; g.ep.out1 = a.dU; g.ep.out2 = a.gH; g.ep.in0 = a.G_save; g.ep.in1 = a.U_save; g.ep.in2 = a.H;
     g.ep.gate = a.gate; g.ep.row_src = a.row_src; g.ep.part = a.part; g.ep.ldo = s.f; g.ep.M_total = (int)M;
     p->prof->begin("gemm_dgrad_down_dswiglu", st);
