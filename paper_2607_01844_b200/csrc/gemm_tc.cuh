@@ -114,7 +114,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// Warp-uniform form: lane 0 waits, the verdict is broadcast, and every lane then observes the
+// Warp-uniform form: lane 0 waits, the outcome is broadcast, and every lane then observes the
 // completed phase itself (so that its later reads are ordered after the barrier).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                int32_t* status, int code, int lane) {
