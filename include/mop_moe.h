@@ -52,12 +52,13 @@ typedef enum { MOP_SCORE_SOFTMAX = 0, MOP_SCORE_SIGMOID = 1 } mop_score_fn;
 typedef enum { MOP_BIAS_NONE = 0, MOP_BIAS_POST_SCORE = 1, MOP_BIAS_PRE_LOGIT = 2 } mop_bias_mode;
 
 /* AUTO: tensor cores when the shape allows, else scalar.  TENSOR: tensor cores or fail.  Both pick
- * per GEMM the schedule measured fastest: forward down-projection (and up-projection when d >= 4096)
- * on the two-CTA tokens-on-N kernel, everything else on the one-CTA kernel (128 x 256 tiles).
+ * per GEMM the schedule measured fastest: the forward down-projection, both data gradients (and the
+ * up-projection when d >= 4096) on the two-CTA tokens-on-N kernel, the weight gradients (and the
+ * up-projection otherwise) on the one-CTA kernel (128 x 256 tiles).
  * The remaining values force one schedule for testing and measurement: TENSOR_1CTA = one-CTA kernel
  * for all token-row GEMMs; TENSOR_2CTA = two-CTA kernel on 256-row pair tiles; TENSOR_MIXED = full
- * pairs on the two-CTA kernel, remaining rows on the one-CTA kernel; TENSOR_TN = both forward GEMMs
- * on the tokens-on-N kernel. */
+ * pairs on the two-CTA kernel, remaining rows on the one-CTA kernel; TENSOR_TN = all four token-row
+ * GEMMs on the tokens-on-N kernel. */
 typedef enum { MOP_GEMM_AUTO = 0, MOP_GEMM_TENSOR = 1, MOP_GEMM_SCALAR = 2, MOP_GEMM_TENSOR_1CTA = 3,
                MOP_GEMM_TENSOR_2CTA = 4, MOP_GEMM_TENSOR_MIXED = 5, MOP_GEMM_TENSOR_TN = 6 } mop_gemm_path;
 
