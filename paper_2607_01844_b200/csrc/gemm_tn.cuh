@@ -316,50 +316,51 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             float v[32];
 
             if constexpr (KIND == TN_F1 || KIND == TN_F1G) {
-                // lanes 0..63 of the CTA hold gate rows, lanes 64..127 the matching up rows
+                // Lanes 0..63 of the CTA hold gate rows, lanes 64..127 the matching up rows: warp q (gate)
+                // and warp q + 2 (up) own the same 32 f columns.  Per chunk of 32 tokens they swap halves
+                // through shared memory (the gate warp hands over G of tokens 16..31, the up warp U of
+                // tokens 0..15), so each evaluates SwiGLU for 16 tokens and writes 16 rows of H.
                 const bool is_up = quarter >= 2;
                 const int fcol = ti.mt * 128 + 64 * (int)rank + 32 * (quarter & 1);   // first f of this warp
                 const bool f_ok = fcol < args.Mw;
-                float* ubuf = reinterpret_cast<float*>(epi_smem + (2 + (quarter & 1)) * 8192);   // in the up warp's region
-                // up warps: [32 x 33 fp32 exchange buffer | one bf16 block]; gate warps: two bf16 blocks
-                uint16_t* st0 = reinterpret_cast<uint16_t*>(is_up ? wbuf + 4352 : wbuf);
-                uint16_t* st1 = st0 + 1024;
+                float* my_x = reinterpret_cast<float*>(wbuf);                                  // 16 x 33 fp32
+                const float* peer_x = reinterpret_cast<const float*>(epi_smem + (quarter ^ 2) * 8192);
+                uint16_t* hb = reinterpret_cast<uint16_t*>(wbuf + 2176);                       // 16 x 32 bf16: H
+                uint16_t* sb = reinterpret_cast<uint16_t*>(wbuf + 3200);                       // 32 x 32 bf16: stash
+                bf16* stash_out = is_up ? args.ep.out2 : args.ep.out1;
+                const int t_own = is_up ? 16 : 0;
                 const int pair_bar = 1 + (quarter & 1);
 #pragma unroll 1
                 for (int c = 0; c < ti.nmma; c += 32) {
                     tmem_ld32(taddr + c, v);
                     const int rows_left = ti.rows - c;
-                    if (is_up) {
 #pragma unroll
-                        for (int tk = 0; tk < 32; ++tk) ubuf[tk * 33 + lane] = v[tk];
-                        if (args.ep.out2) {
+                    for (int i = 0; i < 16; ++i) my_x[i * 33 + lane] = is_up ? v[i] : v[16 + i];
+                    if (stash_out) {
 #pragma unroll
-                            for (int tk = 0; tk < 32; ++tk) st0[tk * 32 + lane] = bf16_bits(v[tk]);
-                        }
-                        bar_pair_sync(pair_bar);     // U is in shared memory
-                        if (args.ep.out2 && f_ok) {
-                            __syncwarp();
-                            tn_write_rows(args.ep.out2, args.ep.ldo, st0, ti.row0 + c, rows_left, fcol, lane);
-                        }
-                        bar_pair_sync(pair_bar);     // the gate warp has read U
-                    } else {
-                        bar_pair_sync(pair_bar);
+                        for (int tk = 0; tk < 32; ++tk) sb[tk * 32 + lane] = bf16_bits(v[tk]);
+                    }
+                    bar_pair_sync(pair_bar);     // both halves are in shared memory
 #pragma unroll
-                        for (int tk = 0; tk < 32; ++tk) {
-                            const float u = ubuf[tk * 33 + lane];
-                            const float g = v[tk];
-                            st0[tk * 32 + lane] = bf16_bits(g * sigmoidf_acc(g) * u);
-                            if (args.ep.out1) st1[tk * 32 + lane] = bf16_bits(g);
-                        }
-                        __syncwarp();
-                        if (f_ok) {
-                            tn_write_rows(args.ep.out0, args.ep.ldo, st0, ti.row0 + c, rows_left, fcol, lane);
-                            if (args.ep.out1)
-                                tn_write_rows(args.ep.out1, args.ep.ldo, st1, ti.row0 + c, rows_left, fcol, lane);
-                        }
-                        bar_pair_sync(pair_bar);
+                    for (int i = 0; i < 16; ++i) {
+                        const float other = peer_x[i * 33 + lane];
+                        const float mine = is_up ? v[16 + i] : v[i];
+                        const float g = is_up ? other : mine, u = is_up ? mine : other;
+                        hb[i * 32 + lane] = bf16_bits(g * sigmoidf_acc(g) * u);
                     }
                     __syncwarp();
+                    if (f_ok) {
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {     // 16 tokens x 32 features of H: 64-byte row segments
+                            const int tok = 8 * i + (lane >> 2), part = lane & 3;
+                            const uint4 hv = *reinterpret_cast<const uint4*>(hb + tok * 32 + part * 8);
+                            if (t_own + tok < rows_left)
+                                *reinterpret_cast<uint4*>(args.ep.out0 + (size_t)(ti.row0 + c + t_own + tok) * args.ep.ldo +
+                                                          fcol + part * 8) = hv;
+                        }
+                        if (stash_out) tn_write_rows(stash_out, args.ep.ldo, sb, ti.row0 + c, rows_left, fcol, lane);
+                    }
+                    bar_pair_sync(pair_bar);     // the partner has read this warp's half
                 }
             } else if constexpr (KIND == TN_B2) {
                 const int fcol = ti.mt * 256 + 128 * (int)rank + 32 * quarter;      // first f column of this warp
