@@ -24,6 +24,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 __device__ __forceinline__ float sigmoidf_acc(float v) { return 1.0f / (1.0f + expf(-v)); }
+// Sigmoid of the SwiGLU epilogues: fast exponential and division (about 2 ulp), far inside the bf16
+// rounding of every value it feeds; all GEMM schedules share it, so they stay bit-identical.  (The
+// router's gates keep the accurate form above.)
+__device__ __forceinline__ float sigmoidf_fast(float v) { return __fdividef(1.0f, 1.0f + __expf(-v)); }
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

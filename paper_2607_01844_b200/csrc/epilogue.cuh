@@ -76,7 +76,7 @@ __device__ __forceinline__ void epi_swiglu(const EpiArgs& ep, int row, int col, 
                                            const float (&u)[C]) {
     float h[C];
 #pragma unroll
-    for (int c = 0; c < C; ++c) h[c] = g[c] * sigmoidf_acc(g[c]) * u[c];
+    for (int c = 0; c < C; ++c) h[c] = g[c] * sigmoidf_fast(g[c]) * u[c];
     const size_t o = (size_t)row * ep.ldo + col;
     store_bf16_run<C>(ep.out0 + o, h);
     if (ep.out1) {
@@ -106,7 +106,7 @@ __device__ __forceinline__ float epi_dh(const EpiArgs& ep, int row, int col, flo
     for (int c = 0; c < C; ++c) {
         dot = fmaf(dhu[c], H[c], dot);
         const float dh = gate * dhu[c];
-        const float s = sigmoidf_acc(G[c]);
+        const float s = sigmoidf_fast(G[c]);
         dG[c] = dh * U[c] * s * (1.0f + G[c] * (1.0f - s));
         dU[c] = dh * (G[c] * s);
         gH[c] = gate * H[c];

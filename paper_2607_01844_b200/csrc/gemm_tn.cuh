@@ -346,7 +346,7 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                         const float other = peer_x[i * 33 + lane];
                         const float mine = is_up ? v[16 + i] : v[i];
                         const float g = is_up ? other : mine, u = is_up ? mine : other;
-                        hb[i * 32 + lane] = bf16_bits(g * sigmoidf_acc(g) * u);
+                        hb[i * 32 + lane] = bf16_bits(g * sigmoidf_fast(g) * u);
                     }
                     __syncwarp();
                     if (f_ok) {
