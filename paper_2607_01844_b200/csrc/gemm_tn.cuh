@@ -369,27 +369,60 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                 const int part = lane & 3;
 #pragma unroll 1
                 for (int c = 0; c < ti.nmma; c += 32) {
-                    tmem_ld32(taddr + c, v);
                     const int rows_left = ti.rows - c;
+                    // the stash (G, U, H: 16 bytes each per lane and sub-block) is requested first, so that its
+                    // latency overlaps the TMEM read and the transposition below
+                    uint4 gq[4], uq[4], hq[4];
+                    float gate[4];
+                    bool ok[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int tok = 8 * i + (lane >> 2);
+                        ok[i] = f_ok && tok < rows_left;
+                        gate[i] = 0.0f;
+                        if (ok[i]) {
+                            const int row = ti.row0 + c + tok;
+                            const size_t o = (size_t)row * args.ep.ldo + fcol + part * 8;
+                            gq[i] = *reinterpret_cast<const uint4*>(args.ep.in0 + o);
+                            uq[i] = *reinterpret_cast<const uint4*>(args.ep.in1 + o);
+                            hq[i] = *reinterpret_cast<const uint4*>(args.ep.in2 + o);
+                            gate[i] = args.ep.gate[args.ep.row_src[row]];
+                        }
+                    }
+                    tmem_ld32(taddr + c, v);
 #pragma unroll
                     for (int tk = 0; tk < 32; ++tk) fbuf[tk * 33 + lane] = v[tk];
                     __syncwarp();
-#pragma unroll 1
+#pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int tok = 8 * i + (lane >> 2);
-                        const bool ok = f_ok && tok < rows_left;
                         float dot = 0.0f;
-                        if (ok) {
-                            const int row = ti.row0 + c + tok;
-                            const float gate = args.ep.gate[args.ep.row_src[row]];
-                            float dhu[8];
+                        if (ok[i]) {
+                            const uint32_t gw[4] = {gq[i].x, gq[i].y, gq[i].z, gq[i].w};
+                            const uint32_t uw[4] = {uq[i].x, uq[i].y, uq[i].z, uq[i].w};
+                            const uint32_t hw[4] = {hq[i].x, hq[i].y, hq[i].z, hq[i].w};
+                            float dG[8], dU[8], gH[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) dhu[j] = fbuf[tok * 33 + part * 8 + j];
-                            dot = epi_dh<8>(args.ep, row, fcol + part * 8, gate, dhu);
+                            for (int j = 0; j < 8; ++j) {
+                                const float G = (j & 1) ? bf16_hi(gw[j >> 1]) : bf16_lo(gw[j >> 1]);
+                                const float U = (j & 1) ? bf16_hi(uw[j >> 1]) : bf16_lo(uw[j >> 1]);
+                                const float H = (j & 1) ? bf16_hi(hw[j >> 1]) : bf16_lo(hw[j >> 1]);
+                                const float dhu = fbuf[tok * 33 + part * 8 + j];
+                                dot = fmaf(dhu, H, dot);
+                                const float dh = gate[i] * dhu;
+                                const float sg = sigmoidf_fast(G);
+                                dG[j] = dh * U * sg * (1.0f + G * (1.0f - sg));
+                                dU[j] = dh * (G * sg);
+                                gH[j] = gate[i] * H;
+                            }
+                            const size_t o = (size_t)(ti.row0 + c + tok) * args.ep.ldo + fcol + part * 8;
+                            store_bf16_run<8>(args.ep.out0 + o, dG);
+                            store_bf16_run<8>(args.ep.out1 + o, dU);
+                            store_bf16_run<8>(args.ep.out2 + o, gH);
                         }
                         dot += __shfl_xor_sync(0xffffffffu, dot, 1);
                         dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                        if (ok && part == 0)
+                        if (ok[i] && part == 0)
                             args.ep.part[(size_t)(fcol >> 5) * args.ep.M_total + ti.row0 + c + tok] = dot;
                     }
                     __syncwarp();
