@@ -169,6 +169,18 @@ def test_gathering_forward_refuses_the_scalar_path():
     assert e.value.code == 6
 
 
+def test_tokens_on_n_kernels_with_three_token_tiles_and_half_filled_k_stages():
+    """700 rows per expert (three token tiles of 240) with d = 320 and f = 192: K is 2.5 and 1.5 pipeline
+    stages of 128, so the last stage of every GEMM is half zero fill; all four token-row GEMMs forced
+    onto the tokens-on-N kernel, compared with the oracle and bit for bit with the one-CTA kernel."""
+    w = synth.small("c2_mid", T=1400, d=320, E=4, k=2, f=192, backward=True, seed=45)
+    _, buf = check_layer(w, binding.GEMM_TENSOR_TN)
+    assert int(buf.counts.max()) > 512
+    _, _, _, ref = run(w, binding.GEMM_TENSOR_1CTA)
+    for n in ("H", "Yp", "Y", "dX", "dW_gate", "dW_up", "dW_down"):
+        assert torch.equal(getattr(buf, n), getattr(ref, n)), n
+
+
 def test_all_keys_equal_goes_to_lowest_ids_and_leaves_experts_empty():
     w = synth.small("c1_tiny", T=96, d=64, E=6, k=2, f=64, backward=True, seed=17)
     host = synth.make_inputs(w, "cpu")
