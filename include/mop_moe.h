@@ -201,7 +201,8 @@ mop_status mop_moe_forward_host(mop_ctx* ctx, const void* x_host, const float* W
  * touch (host_io = 2).  Host buffers must be pinned for the copies to overlap, must stay valid and
  * untouched until mop_host_drain returns, and output buffers of the last TWO calls must be
  * distinct only if the caller reads them before draining.  mop_host_drain makes `stream` wait for
- * every outstanding copy and synchronises it; errors of the kernels surface through mop_poll.
+ * every outstanding copy and synchronises it (call it before mop_destroy too); errors of the kernels
+ * surface through mop_poll.
  * Arguments as in the synchronous forms; results are bit-identical to them. */
 mop_status mop_moe_forward_host_async(mop_ctx* ctx, const void* x_host, const float* W_r, const float* bias,
                                       const void* W_gate, const void* W_up, const void* W_down, void* Y_host,
