@@ -193,9 +193,12 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
     auto decode = [&](int t) {
         TileInfo ti;
-        const int4 m = __ldg(args.mtiles + t / args.tiles_n);
+        int mt, nt;
+        if (args.m_fastest) { const int nm = __ldg(args.n_mtiles); nt = t / nm; mt = t - nt * nm; }
+        else { mt = t / args.tiles_n; nt = t - mt * args.tiles_n; }
+        const int4 m = __ldg(args.mtiles + mt);
         ti.e = m.x; ti.row0 = m.y + 128 * (int)rank; ti.rows = min(128, max(0, m.z - 128 * (int)rank));
-        ti.m0 = 0; ti.nt = t % args.tiles_n; ti.skip = false;
+        ti.m0 = 0; ti.nt = nt; ti.skip = false;
         return ti;
     };
 
@@ -207,7 +210,7 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
                 const TileInfo ti = nxt;
                 if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
-                const int n0 = ti.nt * Tr::N_PER_TILE;
+                const int n0 = ti.nt * Tr::N_PER_TILE + (KIND == TC_VP ? args.n_base : 0);
                 const int nkb = Tr::PHASES * args.kblocks;
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) {
@@ -222,7 +225,8 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
                     tma2_load_2d(sA, ph ? &tmA1 : &tmA0, fb, k0, ti.row0);
                     if constexpr (!Tr::B_MN) {
                         // K-major weights: this CTA's 128 output columns are 128 rows of the [E, N, K] tensor
-                        tma2_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0, n0 + 128 * (int)rank, ti.e);
+                        tma2_load_3d(sB, ph ? &tmB1 : &tmB0, fb, k0 + (KIND == TC_VX ? args.kb_base : 0), n0 + 128 * (int)rank,
+                                     ti.e);
                     } else {
                         // N-major weights: two 64-wide column chunks; with two B tensors (gate | up) the
                         // leader holds the gate columns and the peer the up columns
@@ -236,40 +240,36 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
         }
     } else if (warp == 1) {
         // ===================================================================== MMA issuer (leader CTA)
-        if (leader) {
+        // one thread runs the whole loop (wait, fence, four MMAs, commit) with precomputed descriptors
+        if (leader && lane == 0) {
             constexpr uint32_t idesc = make_idesc2(Tr::B_MN);
+            const uint64_t desc_a = smem_desc(0, 0, 1024);
+            const uint64_t desc_b = Tr::B_MN ? smem_desc(0, TC_CHUNK_BYTES, 1024) : smem_desc(0, 0, 1024);
+            constexpr uint32_t b_step = (Tr::B_MN ? 2048 : 32) >> 4;
             int stage = 0; uint32_t phase = 0; int it = 0; bool alive = true;
+            const int nkb = Tr::PHASES * args.kblocks;
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
                 const int buf = it & 1;
                 const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait_warp(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY, lane))
-                    break;
+                if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * TC_BN;
-                const int nkb = Tr::PHASES * args.kblocks;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait_warp(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL, lane)) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL)) {
                         alive = false; break;
                     }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * T2_STAGE_BYTES;
-                    const uint32_t sB = sA + T2_A_BYTES;
-                    if (lane == 0) {
+                    const uint64_t da = desc_a | (uint64_t)((sA & 0x3ffffu) >> 4);
+                    const uint64_t db = desc_b | (uint64_t)(((sA + T2_A_BYTES) & 0x3ffffu) >> 4);
 #pragma unroll
-                        for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
-                            const uint64_t ad = smem_desc(sA + k4 * 32, 0, 1024);
-                            const uint64_t bd = Tr::B_MN ? smem_desc(sB + k4 * 2048, TC_CHUNK_BYTES, 1024)
-                                                         : smem_desc(sB + k4 * 32, 0, 1024);
-                            umma2_bf16(d_tmem, ad, bd, idesc, (kb | k4) != 0 ? 1u : 0u);
-                        }
-                        umma2_commit_both(empty_bar(stage));
-                    }
-                    __syncwarp();
+                    for (int k4 = 0; k4 < TC_BK / 16; ++k4)
+                        umma2_bf16(d_tmem, da + k4 * 2, db + k4 * b_step, idesc, (kb | k4) != 0 ? 1u : 0u);
+                    umma2_commit_both(empty_bar(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 if (!alive) break;
-                if (lane == 0) umma2_commit_both(tfull_bar(buf));
-                __syncwarp();
+                umma2_commit_both(tfull_bar(buf));
                 ++it;
             }
         }
@@ -287,7 +287,8 @@ tc_gemm2_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
             if (!mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * TC_BN;
-            tc_epilogue_rows<KIND>(args, taddr, r < ti.rows, ti.row0 + r, ti.nt * Tr::N_PER_TILE, ti.nt);
+            tc_epilogue_rows<KIND>(args, taddr, r < ti.rows, ti.row0 + r,
+                                   ti.nt * Tr::N_PER_TILE + (KIND == TC_VP ? args.n_base : 0), ti.nt);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tempty_bar(buf) & T2_PEER_MASK);
@@ -323,6 +324,9 @@ inline mop_status tc2_init() {
     if ((r = tc2_set_smem<TC_F2>()) != MOP_OK) return r;
     if ((r = tc2_set_smem<TC_B2>()) != MOP_OK) return r;
     if ((r = tc2_set_smem<TC_B4>()) != MOP_OK) return r;
+    if ((r = tc2_set_smem<TC_VL>()) != MOP_OK) return r;
+    if ((r = tc2_set_smem<TC_VP>()) != MOP_OK) return r;
+    if ((r = tc2_set_smem<TC_VX>()) != MOP_OK) return r;
     return MOP_OK;
 }
 

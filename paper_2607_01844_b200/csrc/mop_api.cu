@@ -999,6 +999,22 @@ std::mutex g_vocab_mutex;
 TcPlan g_vocab_plan[kMaxDevices];
 Profiler g_vocab_prof;           // never enabled: the plan needs one
 bool g_vocab_ready[kMaxDevices];
+mop_status vocab_plan(int device, TcPlan** out) {
+    TcPlan* p = &g_vocab_plan[device];
+    std::lock_guard<std::mutex> lock(g_vocab_mutex);
+    if (!g_vocab_ready[device]) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MOP_ERR_CUDA;
+        if (prop.major != 10) return MOP_ERR_UNSUPPORTED;
+        mop_moe_shape dummy{};
+        mop_status r = tc_plan_init(p, dummy, prop.multiProcessorCount, &g_vocab_prof);
+        if (r == MOP_OK) r = tc2_init();
+        if (r != MOP_OK) return r;
+        g_vocab_ready[device] = true;
+    }
+    *out = p;
+    return MOP_OK;
+}
 }  // namespace
 
 size_t mop_vocab_workspace_bytes(int32_t N, int32_t H, int32_t V) {
@@ -1019,18 +1035,10 @@ mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const
     if (device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
     DeviceGuard guard(device);
     if (!guard.ok) return MOP_ERR_CUDA;
-    TcPlan* p = &g_vocab_plan[device];
+    TcPlan* p = nullptr;
     {
-        std::lock_guard<std::mutex> lock(g_vocab_mutex);
-        if (!g_vocab_ready[device]) {
-            cudaDeviceProp prop;
-            if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MOP_ERR_CUDA;
-            if (prop.major != 10) return MOP_ERR_UNSUPPORTED;
-            mop_moe_shape dummy{};
-            mop_status r = tc_plan_init(p, dummy, prop.multiProcessorCount, &g_vocab_prof);
-            if (r != MOP_OK) return r;
-            g_vocab_ready[device] = true;
-        }
+        mop_status pr = vocab_plan(device, &p);
+        if (pr != MOP_OK) return pr;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const VocabLayout L = vocab_layout(N, V);
@@ -1043,15 +1051,18 @@ mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const
     const int32_t host_off[2] = {0, N};
     CUDA_OK(cudaMemcpyAsync(off, host_off, sizeof(host_off), cudaMemcpyHostToDevice, st));
     CUDA_OK(cudaMemsetAsync(status, 0, 4, st));
-    tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
+    const bool pair = false;                // measured: the one-CTA kernel is as fast here (online log-sum-exp epilogue)
+    if (pair) tc_build_pairtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
+    else tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
     CUtensorMap mX, mW;
-    if (!tc_map_2d(p, &mX, X, N, H, 128) || !tc_map_chunked_3d(p, &mW, W_voc, 1, H, V, 4)) return MOP_ERR_CUDA;
+    if (!tc_map_2d(p, &mX, X, N, H, 128) || !tc_map_chunked_3d(p, &mW, W_voc, 1, H, V, pair ? 2 : 4)) return MOP_ERR_CUDA;
     TcArgs g{};
     g.offsets = off; g.n_mtiles = tiles; g.mtiles = reinterpret_cast<const int4*>(tiles + 64);
     g.E = 1; g.status = status;
     g.tiles_n = ceil_div(V, 256); g.kblocks = ceil_div(H, TC_BK); g.N = V; g.m_fastest = 1;
     g.targets = targets; g.ylab = ylab; g.ep.part = part; g.ep.M_total = N;
-    mop_status r = tc_launch<TC_VL>(p, "vocab_logits_lse", mX, mX, mW, mW, mX, mX, g, st);
+    mop_status r = pair ? tc2_launch<TC_VL>(p, "vocab_logits_lse", mX, mX, mW, mW, g, st)
+                        : tc_launch<TC_VL>(p, "vocab_logits_lse", mX, mX, mW, mW, mX, mX, g, st);
     if (r != MOP_OK) return r;
     vocab_lse_merge_kernel<<<ceil_div(N, 256), 256, 0, st>>>(reinterpret_cast<const float2*>(part), ylab, loss,
                                                             lse_opt, N, g.tiles_n);
@@ -1073,21 +1084,6 @@ VocabBwdLayout vocab_bwd_layout(int N, int H, int V) {
     L.dx32 = take((size_t)N * H * 4);
     L.total = o;
     return L;
-}
-mop_status vocab_plan(int device, TcPlan** out) {
-    TcPlan* p = &g_vocab_plan[device];
-    std::lock_guard<std::mutex> lock(g_vocab_mutex);
-    if (!g_vocab_ready[device]) {
-        cudaDeviceProp prop;
-        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return MOP_ERR_CUDA;
-        if (prop.major != 10) return MOP_ERR_UNSUPPORTED;
-        mop_moe_shape dummy{};
-        mop_status r = tc_plan_init(p, dummy, prop.multiProcessorCount, &g_vocab_prof);
-        if (r != MOP_OK) return r;
-        g_vocab_ready[device] = true;
-    }
-    *out = p;
-    return MOP_OK;
 }
 }  // namespace
 
@@ -1128,10 +1124,12 @@ mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const
     const int32_t host_off[2] = {0, N};
     CUDA_OK(cudaMemcpyAsync(off, host_off, sizeof(host_off), cudaMemcpyHostToDevice, st));
     CUDA_OK(cudaMemsetAsync(status, 0, 4, st));
-    tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
+    const bool pair = p->sm_count >= 2;     // dY and dX products on the two-CTA kernel (256-row pair tiles)
+    if (pair) tc_build_pairtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
+    else tc_build_mtiles_kernel<<<1, 1024, 0, st>>>(off, 1, reinterpret_cast<int4*>(tiles + 64), tiles);
     CUtensorMap mX, mXT, mWn, mWk;
     if (!tc_map_2d(p, &mX, X, N, H, 128) || !tc_map_chunked_2d(p, &mXT, X, N, H, 2) ||
-        !tc_map_chunked_3d(p, &mWn, W_voc, 1, H, V, 4) || !tc_map_3d(p, &mWk, W_voc, 1, H, V, 256))
+        !tc_map_chunked_3d(p, &mWn, W_voc, 1, H, V, pair ? 2 : 4) || !tc_map_3d(p, &mWk, W_voc, 1, H, V, pair ? 128 : 256))
         return MOP_ERR_CUDA;
     for (int c0 = 0; c0 < V; c0 += L.vc) {
         const int cw = V - c0 < L.vc ? V - c0 : L.vc;
@@ -1146,7 +1144,9 @@ mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const
             TcArgs g = base;
             g.tiles_n = ceil_div(cw, 256); g.kblocks = ceil_div(H, TC_BK); g.N = V; g.m_fastest = 1; g.n_base = c0;
             g.targets = targets; g.row_lse = lse; g.row_g = dloss; g.ep.out0 = dY; g.ep.ldo = L.vc;
-            if ((r = tc_launch<TC_VP>(p, "vocab_dlogits", mX, mX, mWn, mWn, mX, mX, g, st)) != MOP_OK) return r;
+            r = pair ? tc2_launch<TC_VP>(p, "vocab_dlogits", mX, mX, mWn, mWn, g, st)
+                     : tc_launch<TC_VP>(p, "vocab_dlogits", mX, mX, mWn, mWn, mX, mX, g, st);
+            if (r != MOP_OK) return r;
         }
         {   // dW[:, block] = X^T dY (K = the N tokens), written once
             TcArgs g = base;
@@ -1158,7 +1158,9 @@ mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const
             TcArgs g = base;
             g.tiles_n = ceil_div(H, 256); g.kblocks = ceil_div(cw, TC_BK); g.N = H; g.kb_base = c0;
             g.ep.outf = dx32; g.ep.accumulate = c0 > 0 ? 1 : 0;
-            if ((r = tc_launch<TC_VX>(p, "vocab_dgrad", mdYk, mdYk, mWk, mWk, mX, mX, g, st)) != MOP_OK) return r;
+            r = pair ? tc2_launch<TC_VX>(p, "vocab_dgrad", mdYk, mdYk, mWk, mWk, g, st)
+                     : tc_launch<TC_VX>(p, "vocab_dgrad", mdYk, mdYk, mWk, mWk, mX, mX, g, st);
+            if (r != MOP_OK) return r;
         }
     }
     const size_t n8 = (size_t)N * H / 8;
