@@ -35,8 +35,11 @@
 // the tie-break, softmax closed forms for gates, stable argsort for the
 // permutation, a library dense MLP for E=1,k=1, a dense mixture for k=E,
 // automatic differentiation in fp64 and central finite differences for the
-// backward.  Exact float values of the CUDA path beyond the stated tolerance
-// are "parity unpinned" by design.
+// backward; the declared mode against a library restatement in fp64 that rounds
+// at the ten declared tensors (H, the G and U stash, Yp, Y, dG, dU, gate*H,
+// dXp, dX), where removing any one rounding is shown to be detected.  Exact
+// float values of the CUDA path beyond the stated tolerance are "parity
+// unpinned" by design.
 
 #include <algorithm>
 #include <cmath>

@@ -339,6 +339,99 @@ def test_declared_rounding_mode_stays_close_to_exact_mode():
         assert np.array_equal(oracle.bf16_bits_to_f32(synth.bits(torch.from_numpy(b).to(torch.bfloat16))), b)
 
 
+ROUNDING_POINTS = ("H", "G_save", "U_save", "Yp", "Y", "dG", "dU", "gH", "dXp", "dX")
+
+
+def _layer_with_roundings(x, dY, idx, gate, Wg, Wu, Wd, points):
+    """The layer and its backward written with library ops in fp64, rounding to bf16 (nearest even,
+    through the library's own conversion) at exactly the tensors named in `points` and nowhere else.
+    Returns the same outputs as the oracle: Y, G, U, H [T,k,f], Yp [T,k,d], dX, dgate, dW_gate, dW_up, dW_down."""
+    def r(name, v):
+        return v.to(torch.float32).to(torch.bfloat16).to(torch.float64) if name in points else v
+
+    x, dY, Wg, Wu, Wd = (torch.from_numpy(oracle.bf16_bits_to_f64(a)) for a in (x, dY, Wg, Wu, Wd))
+    g_all = torch.from_numpy(gate.astype(np.float64))
+    T, k = idx.shape
+    E, d, f = Wg.shape
+    out = {"Y": torch.zeros(T, d, dtype=torch.float64), "G": torch.zeros(T, k, f, dtype=torch.float64),
+           "U": torch.zeros(T, k, f, dtype=torch.float64), "H": torch.zeros(T, k, f, dtype=torch.float64),
+           "Yp": torch.zeros(T, k, d, dtype=torch.float64), "dX": torch.zeros(T, d, dtype=torch.float64),
+           "dgate": torch.zeros(T, k, dtype=torch.float64), "dW_gate": torch.zeros(E, d, f, dtype=torch.float64),
+           "dW_up": torch.zeros(E, d, f, dtype=torch.float64), "dW_down": torch.zeros(E, f, d, dtype=torch.float64)}
+    for t in range(T):
+        y = torch.zeros(d, dtype=torch.float64)
+        dx = torch.zeros(d, dtype=torch.float64)
+        for j in range(k):
+            e, g = int(idx[t, j]), g_all[t, j]
+            G, U = x[t] @ Wg[e], x[t] @ Wu[e]                    # fp32 accumulators on the device: not rounded
+            H = r("H", torch.nn.functional.silu(G) * U)          # H is made from the unrounded G, U
+            Gs, Us = r("G_save", G), r("U_save", U)              # the stash that the backward reads
+            Yp = r("Yp", g * (H @ Wd[e]))
+            y = y + Yp
+            dHu = Wd[e] @ dY[t]                                  # dY W_down^T, kept in fp32
+            s = torch.sigmoid(Gs)
+            dH = g * dHu
+            dG = r("dG", dH * Us * s * (1 + Gs * (1 - s)))
+            dU = r("dU", dH * (Gs * s))
+            gH = r("gH", g * H)
+            dXp = r("dXp", Wg[e] @ dG + Wu[e] @ dU)
+            dx = dx + dXp
+            out["G"][t, j], out["U"][t, j], out["H"][t, j], out["Yp"][t, j] = Gs, Us, H, Yp
+            out["dgate"][t, j] = dHu @ H
+            out["dW_gate"][e] += torch.outer(x[t], dG)
+            out["dW_up"][e] += torch.outer(x[t], dU)
+            out["dW_down"][e] += torch.outer(gH, dY[t])
+        out["Y"][t] = r("Y", y)
+        out["dX"][t] = r("dX", dx)
+    return {n: v.numpy() for n, v in out.items()}
+
+
+def test_declared_rounding_mode_rounds_at_exactly_the_declared_tensors():
+    """Pin of the declared-rounding mode.  An independent restatement (library ops, fp64, the library's
+    bf16 conversion) that rounds at the ten declared tensors must reproduce every output of the
+    oracle's declared mode to fp32 round-off; the same restatement with any ONE rounding point
+    removed must miss some output by far more than that, so a dropped or misplaced rounding in the
+    oracle cannot pass.  With no rounding point at all it must reproduce the exact mode."""
+    rng = np.random.default_rng(77)
+    T, d, E, k, f = 8, 16, 3, 2, 16
+    x, dY = _rand_bits(rng, (T, d)), _rand_bits(rng, (T, d))
+    Wg, Wu, Wd = (_rand_bits(rng, s, 0.35) for s in ((E, d, f), (E, d, f), (E, f, d)))
+    Wr = (rng.standard_normal((d, E)) * 0.5).astype(np.float32)
+    idx, gate = oracle.route(x, Wr, None, k, 0, 0)
+    ex = np.arange(E, dtype=np.int32)
+
+    def oracle_outputs(declared):
+        Y, G, U, H, Yp = oracle.ffn_fwd(x, idx, gate, Wg, Wu, Wd, declared=declared, want_parts=True)
+        dX, dgate = oracle.ffn_bwd_tokens(x, dY, idx, gate, Wg, Wu, Wd, declared=declared)
+        dWg, dWu, dWd = oracle.ffn_bwd_experts(x, dY, idx, gate, Wg, Wu, Wd, ex, declared=declared)
+        return {"Y": Y, "G": G, "U": U, "H": H, "Yp": Yp, "dX": dX, "dgate": dgate, "dW_gate": dWg, "dW_up": dWu,
+                "dW_down": dWd}
+
+    def worst(a, b):
+        """Largest error over the outputs, each relative to its tensor's largest magnitude."""
+        return max(float(np.max(np.abs(a[n] - b[n])) / max(1.0, np.abs(b[n]).max())) for n in b)
+
+    tol = 1e-6                                            # fp32 accumulation over 16 terms (realised: 5e-8); a bf16 ulp is 4e-3
+    dec = oracle_outputs(True)
+    full = _layer_with_roundings(x, dY, idx, gate, Wg, Wu, Wd, set(ROUNDING_POINTS))
+    for n in dec:
+        err = float(np.max(np.abs(full[n] - dec[n])) / max(1.0, np.abs(dec[n]).max()))
+        assert err <= tol, f"declared mode, {n}: {err:.3e}"
+    none = _layer_with_roundings(x, dY, idx, gate, Wg, Wu, Wd, set())
+    assert worst(none, oracle_outputs(False)) <= tol
+    # the bf16 tensors of the declared mode are representable in bf16
+    for n in ("Y", "G", "U", "H", "Yp", "dX"):
+        assert np.array_equal(oracle.bf16_bits_to_f32(synth.bits(torch.from_numpy(dec[n]).to(torch.bfloat16))), dec[n])
+    # every single rounding point is visible: without it, some output is off by >= 500 x the tolerance
+    for p in ROUNDING_POINTS:
+        without = _layer_with_roundings(x, dY, idx, gate, Wg, Wu, Wd, set(ROUNDING_POINTS) - {p})
+        assert worst(without, dec) >= 500 * tol, f"removing the rounding of {p} goes unnoticed"
+    # and so is a rounding in a place that is not declared: dgate and the weight gradients stay fp32
+    for n in ("dgate", "dW_gate", "dW_up", "dW_down"):
+        as_bf16 = oracle.bf16_bits_to_f32(synth.bits(torch.from_numpy(dec[n].astype(np.float32)).to(torch.bfloat16)))
+        assert np.max(np.abs(as_bf16 - dec[n])) > 500 * tol * max(1.0, np.abs(dec[n]).max()), n
+
+
 # ------------------------------------------------------------------------------ router backward
 @pytest.mark.parametrize("score_fn,bias_mode", [(0, 0), (0, 2), (1, 0), (1, 1), (1, 2)])
 def test_router_backward_matches_automatic_differentiation_of_the_long_form(score_fn, bias_mode):
