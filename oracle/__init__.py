@@ -74,10 +74,9 @@ def f32_to_bf16_bits(a) -> np.ndarray:
     """Round-to-nearest-even fp32 -> bf16 bit patterns, through the oracle's own routine."""
     a = _c(a, np.float32)
     out = np.empty(a.shape, np.uint16)
-    L = lib()
-    flat, o = a.reshape(-1), out.reshape(-1)
-    for i in range(flat.size):
-        o[i] = L.mop_oracle_f32_to_bf16(float(flat[i]))
+    fn = lib().mop_oracle_f32_to_bf16_array
+    fn.restype = None
+    fn(ctypes.c_size_t(a.size), _p(a), _p(out))
     return out
 
 
@@ -238,6 +237,16 @@ def ffn_bwd_experts(x, dY, idx, gate, Wg, Wu, Wd, experts, *, fp64=False, declar
                 _p(dWg), _p(dWu), _p(dWd))
     _check(rc, name)
     return dWg, dWu, dWd
+
+
+def combine(parts, declared=False):
+    """out[n] = sum_j parts[n, j] (fp32, j ascending); declared rounds the sum once to bf16.
+    parts [n,k,d] f32: per-assignment rows, e.g. the Yp of ffn_fwd(want_parts=True)."""
+    parts = _c(parts, np.float32)
+    n, k, d = parts.shape
+    out = np.empty((n, d), np.float32)
+    _check(lib().mop_oracle_combine_f32(n, k, d, int(declared), _p(parts), _p(out)), "combine")
+    return out
 
 
 # ----------------------------------------------------------------------------- router backward

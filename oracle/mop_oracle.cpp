@@ -329,6 +329,10 @@ extern "C" {
 // bf16 helpers exported so that tests can pin the rounding against a library conversion
 uint16_t mop_oracle_f32_to_bf16(float v) { return f32_to_bf16_bits(v); }
 float mop_oracle_bf16_to_f32(uint16_t h) { return bf16_bits_to_f32(h); }
+// the same rounding over an array (one call instead of one per element)
+void mop_oracle_f32_to_bf16_array(size_t n, const float* in, uint16_t* out) {
+    for (size_t i = 0; i < n; ++i) out[i] = f32_to_bf16_bits(in[i]);
+}
 float mop_oracle_sigmoid_contract(float z) { return sigmoid_contract(z); }
 
 // Router: logits, keys, top-k indices and renormalised gates.
@@ -448,6 +452,21 @@ int mop_oracle_permute(int T, int k, int E, const int32_t* idx, int32_t* counts,
         perm_row[a] = p;
         row_src[p] = static_cast<int32_t>(a);
     }
+    return 0;
+}
+
+// Sum over a token's k selected experts, as the layer's definition ends: out[n,:] = sum_j parts[n,j,:],
+// j ascending, in single precision; declared != 0 rounds the sum once to bf16.  parts [n,k,d] holds the
+// per-assignment rows (gate-scaled expert outputs, or per-assignment input gradients).  It lets a test
+// that streams over experts assemble Y and dX of sampled tokens from per-assignment oracle results.
+int mop_oracle_combine_f32(int n, int k, int d, int declared, const float* parts, float* out) {
+    if (n < 0 || k < 1 || d < 1) return 1;
+    for (int q = 0; q < n; ++q)
+        for (int c = 0; c < d; ++c) {
+            float acc = 0.0f;
+            for (int j = 0; j < k; ++j) acc += parts[(static_cast<size_t>(q) * k + j) * d + c];
+            out[static_cast<size_t>(q) * d + c] = maybe_round(acc, declared != 0);
+        }
     return 0;
 }
 

@@ -11,3 +11,13 @@ if str(ROOT) not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Realised float errors of the GPU parity checks: written to gpurun_out/parity_errors.json and summarised."""
+    sys.path.insert(0, str(Path(__file__).resolve().parent))
+    import parity_util
+    table = parity_util.dump()
+    if table:
+        terminalreporter.write_sep("-", "realised parity errors (worst case per tensor)")
+        terminalreporter.write_line(table)

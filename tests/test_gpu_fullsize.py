@@ -1,10 +1,12 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times.
 
 Config 2 is checked on every output element.  Configs 3-5 (11.5-17.3 TFLOP) are checked where the
-oracle can follow in seconds: routing and permutation on ALL tokens (bit-exact), and the float
-outputs on sampled tokens (Y, dX, dgate: the oracle recomputes those tokens through all their
-experts) and sampled experts (dW: the oracle recomputes every row routed to them), plus properties
-that hold at any size.  Inputs are generated on the GPU by the seeded generator and the slices the
+oracle can follow in a minute: routing and permutation on ALL tokens (bit-exact); the float outputs
+Y, dX, dgate on the tokens that own the first and the last row of EVERY live expert (the oracle
+recomputes those tokens through all their experts, streaming the experts' weights); the weight
+gradients of sixteen experts picked by row count (fewest, most, median, just below / above / at
+multiples of 16, 64, 128, and experts whose elements lie beyond 2^31); plus properties that hold at
+any size.  Inputs are generated on the GPU by the seeded generator and the slices the
 oracle needs are downloaded, so both sides see the same bits.
 """
 import numpy as np
@@ -13,7 +15,8 @@ import torch
 
 import oracle
 from paper_2607_01844_b200 import binding, synth
-from test_gpu_parity import MAX_ABS, check_float, check_layer
+from parity_util import check_float
+from test_gpu_parity import check_layer
 
 pytestmark = pytest.mark.gpu
 
@@ -26,30 +29,81 @@ def _np_bias(inp):
     return None if inp["bias"] is None else inp["bias"].cpu().numpy()
 
 
-def _token_problem(w, inp, buf, toks):
-    """Reduced problem holding only the sampled tokens and the experts they use (ids remapped)."""
-    tk = torch.as_tensor(toks, device=buf.idx.device)
-    idx = buf.idx[tk].cpu().numpy()
-    used = np.unique(idx)
-    remap = np.full(w.E, -1, np.int32)
-    remap[used] = np.arange(used.size, dtype=np.int32)
-    ue = torch.as_tensor(used, device=buf.idx.device).long()
-    prob = {"x": synth.bits(inp["x"][tk]), "idx": remap[idx], "gate": buf.gate[tk].cpu().numpy(),
-            "Wg": synth.bits(inp["W_gate"][ue]), "Wu": synth.bits(inp["W_up"][ue]), "Wd": synth.bits(inp["W_down"][ue])}
-    if w.backward:
-        prob["dY"] = synth.bits(inp["dY"][tk])
-    return prob
-
-
-def _expert_problem(w, inp, buf, e):
-    """Reduced problem: every row routed to expert e, as a one-expert top-1 layer."""
-    a = torch.nonzero(buf.idx.reshape(-1) == e).reshape(-1)
+def _expert_problem(w, inp, buf, e, rows=None):
+    """Reduced problem: the rows routed to expert e (all, or the listed assignments), as a one-expert top-1 layer."""
+    a = torch.nonzero(buf.idx.reshape(-1) == e).reshape(-1) if rows is None else rows
     t = a // w.k
-    rows = int(a.numel())
-    return {"rows": rows, "x": synth.bits(inp["x"][t]), "dY": synth.bits(inp["dY"][t]),
-            "idx": np.zeros((rows, 1), np.int32), "gate": buf.gate.reshape(-1)[a].cpu().numpy().reshape(rows, 1),
-            "Wg": synth.bits(inp["W_gate"][e:e + 1]), "Wu": synth.bits(inp["W_up"][e:e + 1]),
-            "Wd": synth.bits(inp["W_down"][e:e + 1])}
+    n = int(a.numel())
+    q = {"rows": n, "x": synth.bits(inp["x"][t]), "idx": np.zeros((n, 1), np.int32),
+         "gate": buf.gate.reshape(-1)[a].cpu().numpy().reshape(n, 1), "Wg": synth.bits(inp["W_gate"][e:e + 1]),
+         "Wu": synth.bits(inp["W_up"][e:e + 1]), "Wd": synth.bits(inp["W_down"][e:e + 1])}
+    if w.backward:
+        q["dY"] = synth.bits(inp["dY"][t])
+    return q
+
+
+def _sampled_tokens(w, offsets, row_src):
+    """Tokens that own the first and the last row of every live expert (at most 2 E of them)."""
+    live = np.nonzero(np.diff(offsets) > 0)[0]
+    rows = np.concatenate([offsets[live], offsets[live + 1] - 1])
+    return np.unique(row_src[rows] // w.k).astype(np.int64)
+
+
+def _oracle_on_sampled_tokens(w, inp, buf, toks, chunk=8):
+    """Y (and dX, dgate) of the sampled tokens in both oracle modes.  The tokens use nearly every expert, so
+    the experts are streamed in chunks: each chunk's weights are downloaded once and its (token, slot) pairs
+    run through the oracle as a top-1 layer over the chunk; oracle.combine then sums a token's k rows."""
+    n = toks.size
+    tk = torch.as_tensor(toks, device=buf.idx.device)
+    idx_s = buf.idx[tk].cpu().numpy()                      # [n, k]
+    gate_s = buf.gate[tk].cpu().numpy()
+    xs = synth.bits(inp["x"][tk])
+    dys = synth.bits(inp["dY"][tk]) if w.backward else None
+    modes = (False, True)
+    Yp = {m: np.zeros((n, w.k, w.d), np.float32) for m in modes}
+    dXp = {m: np.zeros((n, w.k, w.d), np.float32) for m in modes}
+    dg = {m: np.zeros((n, w.k), np.float32) for m in modes}
+    for e0 in range(0, w.E, chunk):
+        e1 = min(w.E, e0 + chunk)
+        q, j = np.nonzero((idx_s >= e0) & (idx_s < e1))    # pairs of this chunk: sampled token q, slot j
+        if q.size == 0:
+            continue
+        sl = slice(e0, e1)
+        Wg, Wu, Wd = (synth.bits(inp[nm][sl]) for nm in ("W_gate", "W_up", "W_down"))
+        pidx = (idx_s[q, j] - e0).astype(np.int32).reshape(-1, 1)
+        pgate = gate_s[q, j].reshape(-1, 1)
+        for m in modes:
+            Yp[m][q, j] = oracle.ffn_fwd(xs[q], pidx, pgate, Wg, Wu, Wd, declared=m)
+            if w.backward:
+                a, b = oracle.ffn_bwd_tokens(xs[q], dys[q], pidx, pgate, Wg, Wu, Wd, declared=m)
+                dXp[m][q, j], dg[m][q, j] = a, b[:, 0]
+    out = {"Y": tuple(oracle.combine(Yp[m], m) for m in modes)}
+    if w.backward:
+        out["dX"] = tuple(oracle.combine(dXp[m], m) for m in modes)
+        out["dgate"] = (dg[False], dg[True])
+    return out
+
+
+def _experts_by_row_count(counts, n_max=16):
+    """Experts whose row counts stress the tile edges: fewest and most rows, the median, the counts just
+    below and just above multiples of 16, 64 and 128, and experts beyond index 146 (whose weight-gradient
+    elements start past 2^31)."""
+    live = np.nonzero(counts > 0)[0]
+    order = live[np.argsort(counts[live], kind="stable")]
+    pick = [int(order[0]), int(order[-1]), int(order[len(order) // 2])]
+    for mod in (128, 64, 16):
+        r = counts[live] % mod
+        pick.append(int(live[np.argmax(r)]))                               # just below a multiple
+        pick.append(int(live[np.argmin(np.where(r == 0, mod, r))]))        # just above a multiple
+        if (r == 0).any():
+            pick.append(int(live[np.argmax(r == 0)]))                      # exactly a multiple
+    high = live[live > 146]
+    pick += [int(e) for e in high[:: max(1, high.size // 5)][:5]] + ([int(high[-1])] if high.size else [])
+    out = []
+    for e in pick:
+        if e not in out:
+            out.append(e)
+    return out[:n_max]
 
 
 @pytest.mark.parametrize("name", ["c3_trillion", "c4_skew", "c5_train"])
@@ -92,25 +146,19 @@ def test_full_size_sampled(name):
         if empty.numel():
             assert torch.all(buf.dW_gate[empty] == 0) and torch.all(buf.dW_down[empty] == 0)
 
-    # ---- float outputs on sampled tokens
-    toks = np.sort(rng.choice(w.T, 5, replace=False)).astype(np.int64)
-    p = _token_problem(w, inp, buf, toks)
+    # ---- float outputs of the tokens that own the first and the last row of EVERY live expert
+    toks = _sampled_tokens(w, offsets, row_src)
+    assert np.unique(idx[toks]).size == int((counts > 0).sum()), "the sample touches every live expert"
     tk = torch.as_tensor(toks, device="cuda")
-    Y_e = oracle.ffn_fwd(p["x"], p["idx"], p["gate"], p["Wg"], p["Wu"], p["Wd"])
-    Y_d = oracle.ffn_fwd(p["x"], p["idx"], p["gate"], p["Wg"], p["Wu"], p["Wd"], declared=True)
-    print(name, "Y", check_float("Y", buf.Y[tk].float().cpu().numpy(), Y_e, Y_d))
+    ref = _oracle_on_sampled_tokens(w, inp, buf, toks)
+    case = f"{name}-full-{toks.size}tok"
+    print(name, check_float("Y", buf.Y[tk].float().cpu().numpy(), *ref["Y"], case))
     if w.backward:
-        scale = lambda a: MAX_ABS * max(1.0, float(np.abs(a).max()))
-        dX_e, dg_e = oracle.ffn_bwd_tokens(p["x"], p["dY"], p["idx"], p["gate"], p["Wg"], p["Wu"], p["Wd"])
-        dX_d, dg_d = oracle.ffn_bwd_tokens(p["x"], p["dY"], p["idx"], p["gate"], p["Wg"], p["Wu"], p["Wd"],
-                                           declared=True)
-        print(name, "dX", check_float("dX", buf.dX[tk].float().cpu().numpy(), dX_e, dX_d, scale(dX_d)))
-        print(name, "dgate", check_float("dgate", buf.dgate[tk].cpu().numpy(), dg_e, dg_d, scale(dg_d)))
-        del p
-        # ---- weight gradients of sampled experts (a light one and a heavy one)
-        order = np.argsort(counts)
-        live = order[counts[order] > 0]
-        for e in (int(live[len(live) // 4]), int(live[-1])):
+        print(name, check_float("dX", buf.dX[tk].float().cpu().numpy(), *ref["dX"], case))
+        print(name, check_float("dgate", buf.dgate[tk].cpu().numpy(), *ref["dgate"], case))
+        del ref
+        # ---- weight gradients of experts picked by row count
+        for e in _experts_by_row_count(counts):
             q = _expert_problem(w, inp, buf, e)
             ex = np.zeros(1, np.int32)
             dW_e = oracle.ffn_bwd_experts(q["x"], q["dY"], q["idx"], q["gate"], q["Wg"], q["Wu"], q["Wd"], ex)
@@ -118,7 +166,8 @@ def test_full_size_sampled(name):
                                           declared=True)
             for nm, got, a, b in zip(("dW_gate", "dW_up", "dW_down"), (buf.dW_gate, buf.dW_up, buf.dW_down), dW_e,
                                      dW_d):
-                print(name, e, q["rows"], nm, check_float(nm, got[e].cpu().numpy(), a[0], b[0], scale(b)))
+                print(name, e, q["rows"], check_float(nm, got[e].cpu().numpy(), a[0], b[0],
+                                                      f"{name}-full-expert{e}-{q['rows']}rows"))
 
 
 def test_full_size_router_backward():

@@ -432,6 +432,56 @@ def test_declared_rounding_mode_rounds_at_exactly_the_declared_tensors():
         assert np.max(np.abs(as_bf16 - dec[n])) > 500 * tol * max(1.0, np.abs(dec[n]).max()), n
 
 
+def test_combine_of_the_per_assignment_rows_is_the_layer_output():
+    """oracle.combine applied to the per-assignment rows reproduces the whole-layer routines bit for bit, in
+    both modes: Y from Yp, and dX of a token from its k one-expert problems (the form the full-size GPU
+    tests use, where the experts of the sampled tokens are streamed)."""
+    x, dY, idx, gate, Wg, Wu, Wd = _setup_bwd(16, T=7, d=12, E=4, k=3, f=16)
+    T, k = idx.shape
+    for declared in (False, True):
+        Y, _, _, _, Yp = oracle.ffn_fwd(x, idx, gate, Wg, Wu, Wd, declared=declared, want_parts=True)
+        assert np.array_equal(oracle.combine(Yp, declared), Y)
+        dX, dgate = oracle.ffn_bwd_tokens(x, dY, idx, gate, Wg, Wu, Wd, declared=declared)
+        parts = np.zeros((T, k, x.shape[1]), np.float32)
+        for t in range(T):
+            for j in range(k):
+                e = int(idx[t, j])
+                one = (x[t:t + 1], dY[t:t + 1], np.zeros((1, 1), np.int32), gate[t:t + 1, j:j + 1], Wg[e:e + 1],
+                       Wu[e:e + 1], Wd[e:e + 1])
+                dXp, dg = oracle.ffn_bwd_tokens(*one, declared=declared)
+                parts[t, j] = dXp[0]
+                assert dg[0, 0] == dgate[t, j]
+        assert np.array_equal(oracle.combine(parts, declared), dX)
+    # closed form: a plain sum, rounded once
+    p3 = np.float32([[[1.0, 2.0 ** -9], [2.0 ** -9, 2.0 ** -9], [0.5, 1.0]]])
+    assert np.array_equal(oracle.combine(p3), np.float32([[1.5 + 2.0 ** -9, 1.0 + 2.0 ** -8]]))
+    assert np.array_equal(oracle.combine(p3, True), np.float32([[1.5, 1.0]]))      # ties go to the even neighbour
+
+
+def test_streamed_assembly_of_sampled_tokens_equals_the_whole_layer_oracle():
+    """The full-size GPU tests assemble the oracle's Y, dX, dgate of sampled tokens from expert chunks;
+    on a small layer that assembly must equal the oracle's whole-layer routines bit for bit."""
+    import types
+
+    from test_gpu_fullsize import _experts_by_row_count, _oracle_on_sampled_tokens, _sampled_tokens
+    w = synth.small("c3_trillion", T=40, d=16, E=11, k=3, f=24, backward=True, seed=5)
+    inp = synth.make_inputs(w, "cpu")
+    xb, dYb, Wg, Wu, Wd = (synth.bits(inp[n]) for n in ("x", "dY", "W_gate", "W_up", "W_down"))
+    idx, gate = oracle.route(xb, inp["W_r"].numpy(), inp["bias"].numpy(), w.k, w.score_fn, w.bias_mode)
+    counts, offsets, perm_row, row_src = oracle.permute(idx, w.E)
+    toks = _sampled_tokens(w, offsets, row_src)
+    assert np.unique(idx[toks]).size == int((counts > 0).sum())
+    buf = types.SimpleNamespace(idx=torch.from_numpy(idx), gate=torch.from_numpy(gate))
+    got = _oracle_on_sampled_tokens(w, inp, buf, toks, chunk=4)
+    for m, declared in enumerate((False, True)):
+        assert np.array_equal(got["Y"][m], oracle.ffn_fwd(xb, idx, gate, Wg, Wu, Wd, declared=declared, toks=toks))
+        dX, dg = oracle.ffn_bwd_tokens(xb, dYb, idx, gate, Wg, Wu, Wd, declared=declared, toks=toks)
+        assert np.array_equal(got["dX"][m], dX) and np.array_equal(got["dgate"][m], dg)
+    picked = _experts_by_row_count(counts)
+    assert len(set(picked)) == len(picked) and all(counts[e] > 0 for e in picked)
+    assert counts[picked[0]] == counts[counts > 0].min() and counts[picked[1]] == counts.max()
+
+
 # ------------------------------------------------------------------------------ router backward
 @pytest.mark.parametrize("score_fn,bias_mode", [(0, 0), (0, 2), (1, 0), (1, 1), (1, 2)])
 def test_router_backward_matches_automatic_differentiation_of_the_long_form(score_fn, bias_mode):
