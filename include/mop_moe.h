@@ -91,6 +91,17 @@ mop_status mop_poll(mop_ctx* ctx, void* stream);
  * mop_poll on this context returns MOP_ERR_TIMEOUT (and clears it).  Nothing faults or traps. */
 mop_status mop_selftest_wait_timeout(mop_ctx* ctx, int64_t limit_cycles, void* stream);
 
+/* Guard bands of the context's workspace (a check that stands in for a memory checker; the paper has no
+ * counterpart).  Every buffer inside the workspace is followed, and the first one preceded, by a
+ * 4 KiB band that no kernel may write.  mop_debug_guard_arm fills the bands with a pattern (enqueued on
+ * `stream`); mop_debug_guard_check synchronises `stream` and returns in *bad_bytes how many band bytes
+ * no longer hold it (0 = no kernel wrote outside its buffers since the bands were armed).
+ * mop_debug_guard_poke overwrites one byte of band number `band` from the host side, so that a test can
+ * see the check respond without any kernel misbehaving. */
+mop_status mop_debug_guard_arm(mop_ctx* ctx, void* stream);
+mop_status mop_debug_guard_check(mop_ctx* ctx, int64_t* bad_bytes, void* stream);
+mop_status mop_debug_guard_poke(mop_ctx* ctx, int32_t band, int32_t byte, void* stream);
+
 /* Number of kernels launched through this context since it was created. */
 int64_t mop_launch_count(const mop_ctx* ctx);
 
@@ -98,7 +109,7 @@ int64_t mop_launch_count(const mop_ctx* ctx);
  * route_bwd) only enqueue work on `stream`: no allocation, no synchronisation, no host read of device
  * data.  A sequence of them may therefore be captured into a CUDA graph and replayed. */
 
-/* Router (Section 2.1: "a lightweight router that sends each token to its top-k experts").
+/* Router of the MoE block (Section 2.1): scores every token against the E experts and keeps its k best.
  *   z[t,e]   = sum_i x[t,i] * W_r[i,e]: one fp32 fused multiply-add per i, i ascending.
  *   key      = z | sigmoid(z) + bias | z + bias       (score_fn, bias_mode)
  *   topk_idx = the k experts with the largest key, descending; equal keys -> lower id.
@@ -144,20 +155,23 @@ mop_status mop_moe_expert_ffn_fwd_gather(mop_ctx* ctx, const void* x, const int3
                                          const int32_t* row_src, const float* topk_gate, const void* W_gate,
                                          const void* W_up, const void* W_down, void* H, void* Yp, void* stream);
 
-/* Unpermute-combine: Y[t,:] = bf16( sum_j Yp[perm_row[t*k+j], :] ), fp32 sum, j ascending.
+/* Unpermute-combine, the last step of the MoE block of Section 2.1 (a token's output is the gate-weighted
+ * sum of its k experts' outputs): Y[t,:] = bf16( sum_j Yp[perm_row[t*k+j], :] ), fp32 sum, j ascending.
  * (The gate was applied by mop_moe_expert_ffn_fwd.)  Also used for dX from dXp.
  * Yp [T*k,d] bf16; perm_row [T*k]; Y [T,d] bf16 out. */
 mop_status mop_moe_combine(mop_ctx* ctx, const void* Yp, const int32_t* perm_row, void* Y, void* stream);
 
-/* Backward of expert_ffn_fwd followed by combine, with topk_idx and topk_gate as inputs of
- * the function (the router's own backward is outside this library).  With p <-> (t,j,e):
+/* Backward of expert_ffn_fwd followed by combine (the paper counts forward and backward compute of every
+ * block, Section 1, and its expert path supports backward gradient propagation, Section 3.3; the formulas
+ * below are the derivative of the forward above), with topk_idx and topk_gate as inputs of the
+ * function (the router's own backward is mop_moe_route_bwd).  With p <-> (t,j,e):
  *   dgate[t,j] = < dY[t,:] W_down[e]^T , H[p,:] >
  *   dH = gate * dY[t,:] W_down[e]^T;  dG = dH * U * s(G) (1 + G (1 - s(G)));  dU = dH * silu(G)
  *   dX[t,:]    = sum_j ( dG[p_j,:] W_gate[e_j]^T + dU[p_j,:] W_up[e_j]^T )
  *   dW_gate[e] = Xp_e^T dG_e;  dW_up[e] = Xp_e^T dU_e;  dW_down[e] = (gate * H_e)^T dY_e
  * dY [T,d] bf16; Xp, G_save, U_save, H, offsets, perm_row, row_src, topk_gate, W_* as above;
  * dX [T,d] bf16 out; dW_gate, dW_up [E,d,f] f32 out; dW_down [E,f,d] f32 out;
- * dgate [T,k] f32 out.  Needs a context created with with_backward >= 1.
+ * dgate [T,k] f32 out.  Needs a context created with with_backward >= 1.  Inputs must be finite.
  * Activation checkpointing (Section 3.1 lists it among the ways to cut transient activation memory):
  * with G_save, U_save and H all NULL (context created with with_backward = 2) the forward may have
  * run without the stash and the up-projection is recomputed here from Xp, bit for bit. */
@@ -259,6 +273,15 @@ mop_status mop_vocab_loss_fwd(int device, int32_t N, int32_t H, int32_t V, const
  * dW_voc [H,V] f32 out (overwritten); workspace: mop_vocab_bwd_workspace_bytes(N, H, V) bytes of
  * device memory, 256-byte aligned, owned by the caller. */
 size_t mop_vocab_bwd_workspace_bytes(int32_t N, int32_t H, int32_t V);
+
+/* The two vocabulary calls have no context, so their kernels record an exhausted device-side wait in the
+ * first word of the caller's workspace.  mop_vocab_poll synchronises `stream`, returns MOP_ERR_TIMEOUT if
+ * the last call that used `workspace` recorded one (its outputs are then not valid) and clears the word.
+ * Check it after a call whose results matter, as mop_poll is checked for a context. */
+mop_status mop_vocab_poll(int device, void* workspace, void* stream);
+/* Self-test of that path, as mop_selftest_wait_timeout: one thread waits `limit_cycles` on a barrier that
+ * nothing completes and records the code in `workspace` (at least 256 bytes); nothing faults or traps. */
+mop_status mop_vocab_selftest_wait_timeout(int device, void* workspace, int64_t limit_cycles, void* stream);
 mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const void* X, const void* W_voc,
                               const int32_t* targets, const float* lse, const float* dloss, void* dX,
                               float* dW_voc, void* workspace, void* stream);

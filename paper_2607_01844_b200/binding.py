@@ -52,6 +52,9 @@ def lib() -> ctypes.CDLL:
         L.mop_poll.argtypes = [_P, _P]
         L.mop_launch_count.argtypes = [_P]
         L.mop_selftest_wait_timeout.argtypes = [_P, ctypes.c_int64, _P]
+        L.mop_debug_guard_arm.argtypes = [_P, _P]
+        L.mop_debug_guard_check.argtypes = [_P, ctypes.POINTER(ctypes.c_int64), _P]
+        L.mop_debug_guard_poke.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, _P]
         L.mop_launch_count.restype = ctypes.c_int64
         L.mop_moe_route.argtypes = [_P] * 8
         L.mop_moe_permute.argtypes = [_P] * 9
@@ -69,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.mop_vocab_workspace_bytes.argtypes = [ctypes.c_int32] * 3
         L.mop_vocab_workspace_bytes.restype = ctypes.c_size_t
         L.mop_vocab_loss_fwd.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 3 + [_P] * 7
+        L.mop_vocab_poll.argtypes = [ctypes.c_int, _P, _P]
+        L.mop_vocab_selftest_wait_timeout.argtypes = [ctypes.c_int, _P, ctypes.c_int64, _P]
         L.mop_vocab_bwd_workspace_bytes.argtypes = [ctypes.c_int32] * 3
         L.mop_vocab_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.mop_vocab_loss_bwd.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 3 + [_P] * 9
@@ -136,6 +141,21 @@ def mop_poll(ctx, stream=None):
 
 def mop_selftest_wait_timeout(ctx, limit_cycles=20_000_000, stream=None):
     _check("mop_selftest_wait_timeout", lib().mop_selftest_wait_timeout(ctx.handle, limit_cycles, _stream(stream)))
+
+
+def mop_debug_guard_arm(ctx, stream=None):
+    _check("mop_debug_guard_arm", lib().mop_debug_guard_arm(ctx.handle, _stream(stream)))
+
+
+def mop_debug_guard_poke(ctx, band, byte, stream=None):
+    _check("mop_debug_guard_poke", lib().mop_debug_guard_poke(ctx.handle, band, byte, _stream(stream)))
+
+
+def mop_debug_guard_check(ctx, stream=None):
+    """Bytes of the workspace's guard bands that were overwritten since they were armed."""
+    bad = ctypes.c_int64(-1)
+    _check("mop_debug_guard_check", lib().mop_debug_guard_check(ctx.handle, ctypes.byref(bad), _stream(stream)))
+    return bad.value
 
 
 def mop_moe_route(ctx, x, W_r, bias, topk_idx, topk_gate, logits=None, stream=None):
@@ -245,6 +265,15 @@ def mop_vocab_loss_fwd(device, X, W_voc, targets, loss, lse=None, workspace=None
            lib().mop_vocab_loss_fwd(device, N, H, V, _ptr(X), _ptr(W_voc), _ptr(targets), _ptr(loss), _ptr(lse),
                                     _ptr(workspace), _stream(stream)))
     return workspace
+
+
+def mop_vocab_poll(device, workspace, stream=None):
+    _check("mop_vocab_poll", lib().mop_vocab_poll(device, _ptr(workspace), _stream(stream)))
+
+
+def mop_vocab_selftest_wait_timeout(device, workspace, limit_cycles=20_000_000, stream=None):
+    _check("mop_vocab_selftest_wait_timeout",
+           lib().mop_vocab_selftest_wait_timeout(device, _ptr(workspace), limit_cycles, _stream(stream)))
 
 
 def mop_vocab_bwd_workspace_bytes(N, H, V):

@@ -612,16 +612,18 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
                 const uint32_t sB = sA + TC_A_BYTES;
                 if constexpr (Tr::RAGGED_K) {
-                    // K tail: rows past the expert's end belong to the next expert.  Zeroing them in
-                    // the A operand alone makes their products vanish (inputs are finite).
+                    // K tail: rows past the expert's end belong to the next expert (or are zero fill).  They are
+                    // cleared in both operands (2 chunks of A and 4 of B, one after the other in the stage), so
+                    // that nothing of a neighbour, not even an Inf or a NaN, can reach this expert's gradient.
                     const int valid = ti.rows - kb * TC_BK;
                     if (valid < TC_BK) {
                         uint8_t* base = smem + stage * TC_STAGE_BYTES;
                         const int n16 = (TC_BK - valid) * 8;     // 16-byte vectors per chunk to clear
                         for (int i = lane; i < n16; i += 32) {
                             const int off = (valid + (i >> 3)) * 128 + (i & 7) * 16;
-                            *reinterpret_cast<uint4*>(base + off) = make_uint4(0, 0, 0, 0);
-                            *reinterpret_cast<uint4*>(base + TC_CHUNK_BYTES + off) = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                            for (int ch = 0; ch < TC_STAGE_BYTES / TC_CHUNK_BYTES; ++ch)
+                                *reinterpret_cast<uint4*>(base + ch * TC_CHUNK_BYTES + off) = make_uint4(0, 0, 0, 0);
                         }
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();

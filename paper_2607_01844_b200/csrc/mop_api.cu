@@ -50,11 +50,20 @@ struct mop_ctx {
     uint64_t host_steps;
     TcPlan plan;
     Profiler prof;
+    unsigned long long guard_off[96];    // guard bands of the workspace (see make_layout)
+    int n_guards;
 };
 
 namespace {
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+// Every region of the workspace is followed (and the first one preceded) by a guard band that no kernel
+// may touch: mop_debug_guard_arm fills the bands with a pattern, mop_debug_guard_check counts the bytes
+// that no longer hold it.  This is how writes past the end of a workspace buffer are caught in tests.
+constexpr size_t GUARD_BYTES = 4096;
+constexpr int MAX_GUARDS = 96;
+constexpr uint32_t GUARD_PATTERN = 0xA5C3A5C3u;
 
 struct Layout {
     size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT, rG, rU, rH;
@@ -62,7 +71,25 @@ struct Layout {
     size_t hG, hU, hdY, hdX, hdgate;
     size_t qx, qY, qidx, qgate, qdY, qdX, qdgate;   // second slot of the pipelined host entry points
     size_t total;
+    size_t guard[MAX_GUARDS];                       // offsets of the guard bands
+    int n_guards;
 };
+
+struct GuardList { unsigned long long off[MAX_GUARDS]; int n; };
+
+__global__ void guard_fill_kernel(char* ws, GuardList g) {
+    uint32_t* band = reinterpret_cast<uint32_t*>(ws + g.off[blockIdx.x]);
+    for (int i = threadIdx.x; i < (int)(GUARD_BYTES / 4); i += blockDim.x) band[i] = GUARD_PATTERN;
+}
+__global__ void guard_check_kernel(const char* ws, GuardList g, unsigned long long* bad) {
+    const uint32_t* band = reinterpret_cast<const uint32_t*>(ws + g.off[blockIdx.x]);
+    int n = 0;
+    for (int i = threadIdx.x; i < (int)(GUARD_BYTES / 4); i += blockDim.x) {
+        const uint32_t x = band[i] ^ GUARD_PATTERN;     // count the bytes that differ
+        n += ((x & 0xffu) != 0) + ((x & 0xff00u) != 0) + ((x & 0xff0000u) != 0) + ((x & 0xff000000u) != 0);
+    }
+    if (n) atomicAdd(bad, (unsigned long long)n);
+}
 
 int perm_units(const mop_moe_shape& s) { return ceil_div(s.T * s.k, PERM_SEG); }
 int part_tiles(const mop_moe_shape& s) { return ceil_div(s.f, 32); }
@@ -70,7 +97,9 @@ int part_tiles(const mop_moe_shape& s) { return ceil_div(s.f, 32); }
 Layout make_layout(const mop_moe_shape& s) {
     Layout L{};
     size_t o = 0;
-    auto take = [&](size_t bytes) { size_t r = o; o += align_up(bytes); return r; };
+    auto band = [&]() { if (L.n_guards < MAX_GUARDS) L.guard[L.n_guards++] = o; o += GUARD_BYTES; };
+    band();
+    auto take = [&](size_t bytes) { size_t r = o; o += align_up(bytes); band(); return r; };
     const size_t T = s.T, d = s.d, E = s.E, k = s.k, f = s.f, M = T * k;
     L.z = take(T * E * 4);
     L.partial = take((size_t)perm_units(s) * E * 4 + 4);
@@ -302,6 +331,8 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         }
     }
     if (cudaMemset(c->status, 0, 256) != cudaSuccess) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
+    c->n_guards = L.n_guards;
+    for (int i = 0; i < L.n_guards; ++i) c->guard_off[i] = L.guard[i];
     if (shape->host_io == 2) {
         bool ok = cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking) == cudaSuccess;
         for (int i = 0; i < 2 && ok; ++i)
@@ -378,6 +409,44 @@ mop_status mop_selftest_wait_timeout(mop_ctx* c, int64_t limit_cycles, void* str
     CUDA_OK(cudaMemcpyAsync(&flag, gave_up, 4, cudaMemcpyDeviceToHost, st));
     CUDA_OK(cudaStreamSynchronize(st));
     return flag == 1 ? MOP_OK : MOP_ERR_CUDA;            // the wait must have given up, not completed
+}
+
+mop_status mop_debug_guard_arm(mop_ctx* c, void* stream) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    GuardList g;
+    g.n = c->n_guards;
+    for (int i = 0; i < g.n; ++i) g.off[i] = c->guard_off[i];
+    guard_fill_kernel<<<g.n, 256, 0, static_cast<cudaStream_t>(stream)>>>(c->ws, g);
+    return after_launch(c);
+}
+
+mop_status mop_debug_guard_poke(mop_ctx* c, int32_t band, int32_t byte, void* stream) {
+    if (!c || band < 0 || band >= c->n_guards || byte < 0 || byte >= (int32_t)GUARD_BYTES) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    CUDA_OK(cudaMemsetAsync(c->ws + c->guard_off[band] + byte, 0, 1, static_cast<cudaStream_t>(stream)));
+    return MOP_OK;
+}
+
+mop_status mop_debug_guard_check(mop_ctx* c, int64_t* bad_bytes, void* stream) {
+    if (!c || !bad_bytes) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GuardList g;
+    g.n = c->n_guards;
+    for (int i = 0; i < g.n; ++i) g.off[i] = c->guard_off[i];
+    unsigned long long* bad = reinterpret_cast<unsigned long long*>(c->status + 16);   // spare words of the status block
+    CUDA_OK(cudaMemsetAsync(bad, 0, 8, st));
+    guard_check_kernel<<<g.n, 256, 0, st>>>(c->ws, g, bad);
+    if (after_launch(c) != MOP_OK) return MOP_ERR_CUDA;
+    unsigned long long host = 0;
+    CUDA_OK(cudaMemcpyAsync(&host, bad, 8, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    *bad_bytes = (int64_t)host;
+    return MOP_OK;
 }
 
 mop_status mop_poll(mop_ctx* c, void* stream) {
@@ -952,9 +1021,12 @@ mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, i
     if (!counts || !offsets) return MOP_ERR_INVALID_ARG;
     if (!aligned16(counts) || !aligned16(offsets)) return MOP_ERR_ALIGN;
     if (T > 0) {
-        if (!x || !topk_idx || !perm_row || !row_src || !Xp) return MOP_ERR_INVALID_ARG;
-        if (!aligned16(x) || !aligned16(topk_idx) || !aligned16(perm_row) || !aligned16(row_src) || !aligned16(Xp))
-            return MOP_ERR_ALIGN;
+        if (!topk_idx || !perm_row || !row_src) return MOP_ERR_INVALID_ARG;
+        if (!aligned16(topk_idx) || !aligned16(perm_row) || !aligned16(row_src)) return MOP_ERR_ALIGN;
+        if (Xp) {                                   // Xp == NULL: tables only, as in mop_moe_permute
+            if (!x) return MOP_ERR_INVALID_ARG;
+            if (!aligned16(x) || !aligned16(Xp)) return MOP_ERR_ALIGN;
+        }
     }
     if (device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
     DeviceGuard guard(device);
@@ -962,19 +1034,25 @@ mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, i
     StaticSetup su;
     mop_status r = static_setup(device, &su);
     if (r != MOP_OK) return r;
+    cudaGetLastError();                             // an error left by an earlier call is not this call's
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = (size_t)PERM_WARPS * E * sizeof(int32_t);
     // Nothing in the scratch has to start at zero: the histogram kernel writes every entry
     // [unit][expert] that the scan and rank kernels read, so a previous call's contents are dead.
-    if (units > 0) perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, M, E);
-    perm_scan_kernel<<<1, 1024, (E + 1) * sizeof(int32_t), st>>>(su.scratch, counts, offsets, units, E);
     if (units > 0) {
-        perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, perm_row,
-                                                                                    row_src, M, E);
-        const int blocks = min(ceil_div(T, 8), su.sm_count * 8);
-        scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, T,
-                                                    k, d / 8);
+        perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, M, E);
+        if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
     }
+    perm_scan_kernel<<<1, 1024, (E + 1) * sizeof(int32_t), st>>>(su.scratch, counts, offsets, units, E);
+    if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
+    if (units == 0) return MOP_OK;
+    perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, perm_row, row_src,
+                                                                                M, E);
+    if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
+    if (!Xp) return MOP_OK;
+    const int blocks = min(ceil_div(T, 8), su.sm_count * 8);
+    scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, T, k,
+                                                d / 8);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
@@ -987,9 +1065,9 @@ VocabLayout vocab_layout(int N, int V) {
     VocabLayout L{};
     size_t o = 0;
     auto take = [&](size_t b) { size_t r = o; o += align_up(b); return r; };
+    L.status = take(256);                 // first: mop_vocab_poll reads it without knowing the shape
     L.off = take(16);
     L.tiles = take(tc_tile_table_bytes(N, 1));
-    L.status = take(256);
     L.ylab = take((size_t)N * 4);
     L.part = take((size_t)ceil_div(V, 256) * N * 8);
     L.total = o;
@@ -1077,15 +1155,49 @@ VocabBwdLayout vocab_bwd_layout(int N, int H, int V) {
     size_t o = 0;
     auto take = [&](size_t b) { size_t r = o; o += align_up(b); return r; };
     L.vc = V < kVocabBlock ? V : kVocabBlock;
+    L.status = take(256);                 // first, as in the forward's workspace
     L.off = take(16);
     L.tiles = take(tc_tile_table_bytes(N, 1));
-    L.status = take(256);
     L.dy = take((size_t)N * L.vc * 2);
     L.dx32 = take((size_t)N * H * 4);
     L.total = o;
     return L;
 }
 }  // namespace
+
+mop_status mop_vocab_poll(int device, void* workspace, void* stream) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MOP_ERR_INVALID_ARG;
+    if (device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;   // both vocabulary workspaces start with their status block
+    CUDA_OK(cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    if (word != 0) {
+        CUDA_OK(cudaMemsetAsync(workspace, 0, 4, st));
+        CUDA_OK(cudaStreamSynchronize(st));
+        return MOP_ERR_TIMEOUT;
+    }
+    return MOP_OK;
+}
+
+mop_status mop_vocab_selftest_wait_timeout(int device, void* workspace, int64_t limit_cycles, void* stream) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MOP_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > 4000000000ll || device < 0 || device >= kMaxDevices) return MOP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* status = static_cast<int32_t*>(workspace);
+    int32_t* gave_up = status + 8;                       // a spare word of the status block
+    CUDA_OK(cudaMemsetAsync(gave_up, 0, 4, st));
+    tc_wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_cycles, gave_up);
+    if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
+    int32_t flag = 0;
+    CUDA_OK(cudaMemcpyAsync(&flag, gave_up, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    return flag == 1 ? MOP_OK : MOP_ERR_CUDA;
+}
 
 size_t mop_vocab_bwd_workspace_bytes(int32_t N, int32_t H, int32_t V) {
     if (N < 0 || H < 64 || V < 64 || H % 64 || V % 64) return 0;
@@ -1164,7 +1276,8 @@ mop_status mop_vocab_loss_bwd(int device, int32_t N, int32_t H, int32_t V, const
         }
     }
     const size_t n8 = (size_t)N * H / 8;
-    f32_to_bf16_kernel<<<(unsigned)((n8 + 255) / 256 < 148 * 16 ? (n8 + 255) / 256 : 148 * 16), 256, 0, st>>>(
+    const size_t cap = (size_t)p->sm_count * 16;
+    f32_to_bf16_kernel<<<(unsigned)((n8 + 255) / 256 < cap ? (n8 + 255) / 256 : cap), 256, 0, st>>>(
         reinterpret_cast<const float4*>(dx32), static_cast<uint4*>(dX), n8);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }

@@ -1,5 +1,5 @@
-// Router kernels: exact fp32 scoring and warp-per-token top-k with gate renormalisation.
-// Section 2.1 of the paper ("a lightweight router that sends each token to its top-k experts").
+// Router kernels: exact fp32 scoring and warp-per-token top-k with gate renormalisation
+// (the router of the MoE block, Section 2.1 of the paper).
 #pragma once
 #include "common.cuh"
 
@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) route_select_kernel(const floa
     }
     __syncwarp();
     uint32_t taken = 0;
-    float my_z = 0.0f;     // lane j keeps the gate logit of the j-th pick (k <= 32) ...
+    float my_z = 0.0f;     // lane j keeps the gate logit and the id of the j-th pick (k <= 32, checked on the host)
     int my_e = 0;
     for (int j = 0; j < k; ++j) {
         int best = -1;
@@ -258,46 +258,27 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) route_select_kernel(const floa
         }
         // every lane now holds the same winner (the comparison is a total order on (key, id))
         if ((best & 31) == lane) taken |= 1u << (best >> 5);
-        if ((j & 31) == lane) {
-            // picks beyond 32 are handled in a second pass below (k <= 32 in every workload)
+        if (j == lane) {
             my_e = best;
             my_z = zg[best];
         }
-        if (k > 32 && lane == 0) idx[(size_t)t * k + j] = best;
     }
-    if (k <= 32) {
-        const bool act = lane < k;
-        float s;
-        if (score_fn == 0) {
-            float m = act ? my_z : -INFINITY;
+    const bool act = lane < k;
+    float s;
+    if (score_fn == 0) {
+        float m = act ? my_z : -INFINITY;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-            s = act ? expf(my_z - m) : 0.0f;
-        } else {
-            s = act ? sigmoidf_acc(my_z) : 0.0f;
-        }
-        float sum = s;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        if (act) {
-            idx[(size_t)t * k + lane] = my_e;
-            gate[(size_t)t * k + lane] = s / sum;
-        }
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        s = act ? expf(my_z - m) : 0.0f;
     } else {
-        // generic tail (k > 32): lane 0 recomputes the gates from the stored indices
-        __syncwarp();
-        if (lane == 0) {
-            float m = -INFINITY, sum = 0.0f;
-            for (int j = 0; j < k; ++j) m = fmaxf(m, zg[idx[(size_t)t * k + j]]);
-            for (int j = 0; j < k; ++j) {
-                const float zz = zg[idx[(size_t)t * k + j]];
-                sum += (score_fn == 0) ? expf(zz - m) : sigmoidf_acc(zz);
-            }
-            for (int j = 0; j < k; ++j) {
-                const float zz = zg[idx[(size_t)t * k + j]];
-                gate[(size_t)t * k + j] = ((score_fn == 0) ? expf(zz - m) : sigmoidf_acc(zz)) / sum;
-            }
-        }
+        s = act ? sigmoidf_acc(my_z) : 0.0f;
+    }
+    float sum = s;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (act) {
+        idx[(size_t)t * k + lane] = my_e;
+        gate[(size_t)t * k + lane] = s / sum;
     }
 }
 
