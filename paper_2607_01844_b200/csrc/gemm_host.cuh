@@ -136,8 +136,8 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
         !tc_map_2d(p, &mdG, a.dG, M, s.f, 128) || !tc_map_2d(p, &mdU, a.dU, M, s.f, 128) ||
         !tc_map_3d(p, &mWgK, a.W_gate, s.E, s.d, s.f, 256) || !tc_map_3d(p, &mWuK, a.W_up, s.E, s.d, s.f, 256) ||
         !tc_map_chunked_2d(p, &mgH, a.gH, M, s.f, 2) || !tc_map_chunked_2d(p, &mdYpB, a.dYp, M, s.d, 4) ||
-        !tc_map_chunked_2d(p, &mXpA, a.Xp, M, s.d, 2) || !tc_map_chunked_2d(p, &mdGB, a.dG, M, s.f, 2) ||
-        !tc_map_chunked_2d(p, &mdUB, a.dU, M, s.f, 2))
+        !tc_map_chunked_2d(p, &mXpA, a.Xp, M, s.d, 2) || !tc_map_chunked_2d(p, &mdGB, a.dG, M, s.f, 4) ||
+        !tc_map_chunked_2d(p, &mdUB, a.dU, M, s.f, 4))
         return MOP_ERR_CUDA;
     int32_t* ttiles = tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4);
     if (p->fwd_tn & 12) {
@@ -175,9 +175,9 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
         if ((r = tc_launch<TC_WD>(p, "gemm_wgrad_down", mgH, mgH, mdYpB, mdYpB, moWd, moWd, g, st)) != MOP_OK) return r;
         ++*launches;
     }
-    {   // WGU: [dW_gate | dW_up][e] = Xp_e^T [dG | dU]_e
+    {   // WGU: dW_gate[e] = Xp_e^T dG_e and dW_up[e] = Xp_e^T dU_e: per m-block the n-tiles of dW_gate, then those of dW_up
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
-        g.tiles_n = ceil_div(s.f, 128); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
+        g.tiles_n = 2 * ceil_div(s.f, 256); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
         g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate;
         if ((r = tc_launch<TC_WGU>(p, "gemm_wgrad_gate_up", mXpA, mXpA, mdGB, mdUB, moWg, moWu, g, st)) != MOP_OK) return r;
         ++*launches;

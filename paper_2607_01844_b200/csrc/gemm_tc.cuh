@@ -7,7 +7,7 @@
 //   B2   dHu   = dYp W_down[e]^T                  SwiGLU-backward epilogue            ragged M
 //   B4   dXp   = dG W_gate[e]^T + dU W_up[e]^T    (two K phases)  -> bf16             ragged M
 //   WD   dW_down[e] = (gate H)_e^T dYp_e          fp32 store                          ragged K
-//   WGU  [dW_gate|dW_up][e] = Xp_e^T [dG|dU]_e    fp32 store                          ragged K
+//   WGU  dW_gate[e] = Xp_e^T dG_e, dW_up[e] = Xp_e^T dU_e  (a tile belongs to one of the two)  ragged K
 //   VL   Y = X W_voc (never stored)               online log-sum-exp partials         dense M
 //   VP   dY = g ([v = t] - exp(X W_voc - lse))     bf16, one block of vocabulary columns dense M
 //   VX   dX += dY W_voc^T over that block          fp32 read-modify-write              dense M
@@ -40,7 +40,11 @@ template <int KIND>
 struct TcTraits {
     static constexpr bool A_MN = (KIND == TC_WD || KIND == TC_WGU);   // A is M-contiguous in memory
     static constexpr bool B_MN = (KIND != TC_B2 && KIND != TC_B4 && KIND != TC_VX);   // B is N-contiguous in memory
-    static constexpr bool DUAL_B = (KIND == TC_F1 || KIND == TC_WGU); // two B tensors, 128 columns each
+    static constexpr bool DUAL_B = (KIND == TC_F1);                   // two B tensors, 128 columns each
+    // Both weight gradients of the up-projection in one launch: the second half of an m-block's n-tiles takes
+    // its B operand from the second tensor (dU) and writes the second output (dW_up).  A tile thus covers 256
+    // columns (1 KiB per row) of ONE gradient: DRAM takes such a store stream faster than 2 x 512 bytes.
+    static constexpr bool SEL_B = (KIND == TC_WGU);
     static constexpr bool RAGGED_K = A_MN;
     static constexpr bool B_WEIGHT = !RAGGED_K;                       // B is an [E, ., .] weight tensor
     static constexpr int PHASES = (KIND == TC_B4) ? 2 : 1;
@@ -112,6 +116,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+
+// Barrier over `nthreads` threads (named barrier `id`) that also ANDs a predicate: every participant
+// learns whether ALL of them arrived with ok.  Used where warps that took a bounded wait separately
+// must agree on giving up before they meet at plain barriers (a warp that left alone would hang the rest).
+__device__ __forceinline__ bool bar_vote_all(int id, int nthreads, bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\nsetp.ne.b32 p, %3, 0;\nbar.red.and.pred q, %1, %2, p;\nselp.u32 %0, 1, 0, q;\n}"
+        : "=r"(r)
+        : "r"(id), "r"(nthreads), "r"(ok ? 1u : 0u)
+        : "memory");
+    return r != 0;
 }
 
 // Warp-uniform form: lane 0 waits, the outcome is broadcast, and every lane then observes the
@@ -260,6 +277,12 @@ __device__ __forceinline__ void tmem_ld_wait(float (&a)[32], float (&b)[32]) {
     for (int i = 0; i < 32; ++i) asm volatile("" : "+f"(a[i]), "+f"(b[i]));
 }
 
+__device__ __forceinline__ void tmem_ld_wait4(float (&a)[32], float (&b)[32], float (&c)[32], float (&d)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) asm volatile("" : "+f"(a[i]), "+f"(b[i]), "+f"(c[i]), "+f"(d[i]));
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (Blackwell).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
@@ -296,18 +319,24 @@ struct TileInfo {
     int e, row0, rows;   // ragged M: first global row and valid rows; ragged K: first k row and k count
     int m0;              // ragged K: first output row of the tile inside the expert's matrix
     int nt;              // n-tile index
+    int sel;             // SEL_B kinds: 1 = second B tensor and second output
     bool skip;           // nothing to multiply (expert without rows)
 };
 
 template <int KIND>
 __device__ __forceinline__ TileInfo decode_tile(const TcArgs& a, int t) {
     TileInfo ti;
+    ti.sel = 0;
     if constexpr (TcTraits<KIND>::RAGGED_K) {
         const int per_e = a.tiles_m_fixed * a.tiles_n;
         ti.e = t / per_e;
         const int r = t - ti.e * per_e;
         ti.m0 = (r / a.tiles_n) * TC_BM;
         ti.nt = r % a.tiles_n;
+        if constexpr (TcTraits<KIND>::SEL_B) {
+            const int half_n = a.tiles_n >> 1;
+            if (ti.nt >= half_n) { ti.nt -= half_n; ti.sel = 1; }
+        }
         ti.row0 = __ldg(a.offsets + ti.e);
         ti.rows = __ldg(a.offsets + ti.e + 1) - ti.row0;
         ti.skip = ti.rows <= 0;
@@ -491,7 +520,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB0);
         if (Tr::PHASES == 2) tma_prefetch_desc(&tmA1);
-        if (Tr::DUAL_B || Tr::PHASES == 2) tma_prefetch_desc(&tmB1);
+        if (Tr::DUAL_B || Tr::SEL_B || Tr::PHASES == 2) tma_prefetch_desc(&tmB1);
     }
     if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
@@ -543,8 +572,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                             if constexpr (Tr::DUAL_B) tma_load_4d(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, k0, n0 >> 6, ti.e);
                         } else {
                             const int krow = ti.row0 + kb * TC_BK;
-                            tma_load_3d_hint(sB, &tmB0, fb, 0, krow, n0 >> 6, keep);
-                            if constexpr (Tr::DUAL_B) tma_load_3d_hint(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, krow, n0 >> 6, keep);
+                            tma_load_3d_hint(sB, (Tr::SEL_B && ti.sel) ? &tmB1 : &tmB0, fb, 0, krow, n0 >> 6, keep);
                         }
                     }
                     if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
@@ -611,27 +639,31 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 tc_fence_after();
                 const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
                 const uint32_t sB = sA + TC_A_BYTES;
+                int n_k4 = TC_BK / 16;                   // MMAs (16 rows of K each) of this block
                 if constexpr (Tr::RAGGED_K) {
-                    // K tail: rows past the expert's end belong to the next expert (or are zero fill).  They are
-                    // cleared in both operands (2 chunks of A and 4 of B, one after the other in the stage), so
-                    // that nothing of a neighbour, not even an Inf or a NaN, can reach this expert's gradient.
+                    // K tail: rows past the expert's end belong to the next expert (or are zero fill).  Whole
+                    // groups of 16 such rows are simply not multiplied; the rest of the last group (at most 15
+                    // rows) is cleared in both operands (2 chunks of A and 4 of B, one after the other in the
+                    // stage), so that nothing of a neighbour, not even an Inf or a NaN, reaches this gradient.
                     const int valid = ti.rows - kb * TC_BK;
                     if (valid < TC_BK) {
+                        n_k4 = (valid + 15) >> 4;
                         uint8_t* base = smem + stage * TC_STAGE_BYTES;
-                        const int n16 = (TC_BK - valid) * 8;     // 16-byte vectors per chunk to clear
+                        const int n16 = (n_k4 * 16 - valid) * 8; // 16-byte vectors per chunk to clear
                         for (int i = lane; i < n16; i += 32) {
                             const int off = (valid + (i >> 3)) * 128 + (i & 7) * 16;
 #pragma unroll
                             for (int ch = 0; ch < TC_STAGE_BYTES / TC_CHUNK_BYTES; ++ch)
                                 *reinterpret_cast<uint4*>(base + ch * TC_CHUNK_BYTES + off) = make_uint4(0, 0, 0, 0);
                         }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        if (n16 > 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
                     }
                 }
                 if (lane == 0) {
 #pragma unroll
                     for (int k4 = 0; k4 < TC_BK / 16; ++k4) {
+                        if (k4 >= n_k4) break;
                         const uint64_t ad = Tr::A_MN ? smem_desc(sA + k4 * 2048, mn_lbo, mn_sbo)
                                                      : smem_desc(sA + k4 * 32, 0, 1024);
                         const uint64_t bd = Tr::B_MN ? smem_desc(sB + k4 * 2048, mn_lbo, mn_sbo)
@@ -665,18 +697,19 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                     // expert without rows: its gradient is zero (or unchanged when accumulating)
                     if (!args.ep.accumulate && half == 0 && ti.m0 + r < args.Mfix) {
                         const size_t ro = ((size_t)ti.e * args.Mfix + ti.m0 + r) * args.N;
-                        for (int c = 0; c < TC_BN; c += 4) {
-                            const int cc = Tr::DUAL_B ? (c & 127) : c;
-                            float* dst = (Tr::DUAL_B && c >= 128) ? args.outf1 : args.ep.outf;
-                            if (n0 + cc < args.N) *reinterpret_cast<float4*>(dst + ro + n0 + cc) = make_float4(0, 0, 0, 0);
-                        }
+                        float* dst = (Tr::SEL_B && ti.sel) ? args.outf1 : args.ep.outf;
+                        for (int c = 0; c < TC_BN; c += 4)
+                            if (n0 + c < args.N) *reinterpret_cast<float4*>(dst + ro + n0 + c) = make_float4(0, 0, 0, 0);
                     }
                     continue;
                 }
             }
             const int buf = it & 1;
             const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
-            if (!mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane)) break;
+            bool ready = mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane);
+            // the four warps of a column half meet at named barriers below: they give up together or not at all
+            if constexpr (Tr::RAGGED_K) ready = bar_vote_all(1 + half, 128, ready);
+            if (!ready) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * TC_BN;
             const bool row_ok = Tr::RAGGED_K ? (ti.m0 + r < args.Mfix) : (r < ti.rows);
@@ -687,48 +720,51 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             if constexpr (!Tr::RAGGED_K) {
                 tc_epilogue_rows<KIND>(args, taddr, row_ok, grow, n0, ti.nt);
             } else {
-                // Weight-gradient tile: the four warps of a column half stage 128 rows x 32 fp32 columns
-                // in shared memory (128-byte rows, 16-byte chunks XOR-swizzled by row: the layout of a
-                // 128B-swizzle tensor map, conflict-free for one-row-per-lane writes) and one thread hands
-                // the 16 KiB box to TMA, which writes whole 128-byte lines and clips rows >= Mfix and
-                // columns >= N.  Only the box writes use the load/store pipe.  Two boxes per half.
+                // Weight-gradient tile.  Each warp first reads its 32 rows x 128 columns from TMEM in one go and
+                // hands the accumulator back, so that the MMA warp can run two tiles ahead of the stores.  Then
+                // the four warps of a column half stage 128 rows x 32 fp32 columns in shared memory (128-byte
+                // rows, 16-byte chunks XOR-swizzled by row: the layout of a 128B-swizzle tensor map,
+                // conflict-free for one-row-per-lane writes) and one thread hands the 16 KiB box to TMA, which
+                // writes whole 128-byte lines and clips rows >= Mfix and columns >= N.  Two boxes per half.
                 uint8_t* gbase = smem + TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + half * 32768;
-                const CUtensorMap* mo = (Tr::DUAL_B && half) ? &tmO1 : &tmO0;
+                const CUtensorMap* mo = (Tr::SEL_B && ti.sel) ? &tmO1 : &tmO0;
                 const bool issuer = (quarter == 0 && lane == 0);
                 const uint64_t stream_out = l2_policy_evict_first();
                 const int gbar = 1 + half;               // named barrier of this half's 128 threads
-                float acc_b[32];
-#pragma unroll 1
-                for (int c = half * 128; c < half * 128 + 128; c += 64) {
-                    tmem_ld32_nowait(taddr + c, acc);
-                    tmem_ld32_nowait(taddr + c + 32, acc_b);
-                    tmem_ld_wait(acc, acc_b);
+                float a0[32], a1[32], a2[32], a3[32];
+                tmem_ld32_nowait(taddr + half * 128, a0);
+                tmem_ld32_nowait(taddr + half * 128 + 32, a1);
+                tmem_ld32_nowait(taddr + half * 128 + 64, a2);
+                tmem_ld32_nowait(taddr + half * 128 + 96, a3);
+                tmem_ld_wait4(a0, a1, a2, a3);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint8_t* box = gbase + (sbuf & 1) * 16384;
-                        if (issuer) tma_store_wait_read<1>();     // the box staged two steps ago has been read
-                        asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
-                        uint8_t* rowp = box + (quarter * 32 + lane) * 128;
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint8_t* box = gbase + (sbuf & 1) * 16384;
+                    if (issuer) tma_store_wait_read<1>();     // the box staged two steps ago has been read
+                    asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
+                    uint8_t* rowp = box + (quarter * 32 + lane) * 128;
+                    const float(&v)[32] = cc == 0 ? a0 : cc == 1 ? a1 : cc == 2 ? a2 : a3;
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 v = h ? make_float4(acc_b[4 * j], acc_b[4 * j + 1], acc_b[4 * j + 2], acc_b[4 * j + 3])
-                                               : make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
-                            *reinterpret_cast<float4*>(rowp + ((j ^ (lane & 7)) << 4)) = v;
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<float4*>(rowp + ((j ^ (lane & 7)) << 4)) =
+                            make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
+                    if (issuer) {
+                        const int gcol = n0 + half * 128 + 32 * cc;
+                        if (gcol < args.N) {
+                            if (args.ep.accumulate) tma_reduce_add_3d(mo, smem_u32(box), gcol, ti.m0, ti.e);
+                            else tma_store_3d_hint(mo, smem_u32(box), gcol, ti.m0, ti.e, stream_out);
                         }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
-                        if (issuer) {
-                            const int col = c + 32 * h;
-                            const int gcol = n0 + (Tr::DUAL_B ? (col & 127) : col);
-                            if (gcol < args.N) {
-                                if (args.ep.accumulate) tma_reduce_add_3d(mo, smem_u32(box), gcol, ti.m0, ti.e);
-                                else tma_store_3d_hint(mo, smem_u32(box), gcol, ti.m0, ti.e, stream_out);
-                            }
-                            tma_store_commit();
-                        }
-                        ++sbuf;
+                        tma_store_commit();
                     }
+                    ++sbuf;
                 }
+                ++it;
+                continue;
             }
             tc_fence_before();
             __syncwarp();
