@@ -53,6 +53,12 @@ def peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+def config_of(w):
+    """The workload as both arms print it."""
+    return {"workload": w.name, "T": w.T, "d": w.d, "E": w.E, "k": w.k, "f": w.f,
+            "pass": "fwd+bwd" if w.backward else "fwd", "l2": "inputs larger than L2"}
+
+
 def flops_per_step(w):
     return (18 if w.backward else 6) * w.M * w.d * w.f
 
@@ -197,7 +203,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": "moe_layer_tflops", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "T": w.T, "d": w.d, "E": w.E, "k": w.k, "f": w.f},
+        "config": config_of(w),
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -267,45 +273,13 @@ def run_vocab(args):
 
 
 # --------------------------------------------------------------------------------------- CUDA path
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None)
-    ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c5_train", choices=sorted(synth.WORKLOADS) + ["vocab_loss", "vocab_train"])
-    ap.add_argument("--shape", default=None,
-                    help="T,d,E,k,f overriding the named workload's sizes (same distributions): small cases for "
-                         "profiler captures")
-    ap.add_argument("--gemm-path", type=int, default=0, help="mop_gemm_path (0 = library default)")
-    ap.add_argument("--with-router-bwd", action="store_true",
-                    help="also run the router backward (dgate -> dW_r, dX) in every step of a fwd+bwd workload")
-    ap.add_argument("--gather", action="store_true",
-                    help="forward-only workloads: up-projection gathers its rows from x (no permuted copy)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    if args.workload in ("vocab_loss", "vocab_train"):
-        return run_vocab(args)
-    w = synth.WORKLOADS[args.workload]
-    if args.shape:
-        T, d, E, k, f = (int(v) for v in args.shape.split(","))
-        import dataclasses
-        w = dataclasses.replace(w, T=T, d=d, E=E, k=k, f=f, name=f"{w.name}[{args.shape}]")
-    if args.impl == "reference":
-        args.steps = args.steps or 3
-        args.warmup = 1 if args.warmup is None else args.warmup
-        return run_reference(args, w)
-    args.steps = args.steps or 20
-    args.warmup = max(3, args.warmup or 3)
-
+def bench_workload(w, args, steps, warmup, with_cpu_baseline):
+    """One workload on this rank's GPU: device-resident timing with a per-kernel profile, the end-to-end
+    host-buffer timing, the roofline of the dominant kernel and (optionally) the CPU baseline.  Returns the
+    JSON record (rank 0) or None."""
     from paper_2607_01844_b200 import binding
     rank, local, world = launch.env_world()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
-    torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    launch.init("nccl", dev)
     barrier = launch.barrier
 
     inp = synth.make_inputs(w, dev)
@@ -334,7 +308,7 @@ def main():
             binding.mop_moe_route_bwd(ctx, logits, inp["bias"], buf.idx, buf.gate, buf.dgate, buf.Xp, buf.offsets,
                                       buf.perm_row, inp["W_r"], dW_r, None, buf.dX, stream)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step()
     binding.mop_poll(ctx, stream)
     binding.mop_profile_enable(ctx, True)
@@ -344,7 +318,7 @@ def main():
     sampler.start()
     l0 = ctx.launch_count
     ev0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(steps):
         step()
     ev1.record(stream)
     torch.cuda.synchronize(); barrier()
@@ -355,7 +329,7 @@ def main():
     binding.mop_profile_enable(ctx, False)
     binding.mop_poll(ctx, stream)
     ms = launch.max_over_ranks(ms, dev)
-    ms_step = ms / args.steps
+    ms_step = ms / steps
     value = launch.job_throughput(flops_per_step(w), ms_step, world) / 1e12
 
     # ---- end to end through the host-buffer entry point
@@ -389,7 +363,7 @@ def main():
         for _ in range(2):
             host_step()
         binding.mop_host_drain(ctx, stream)
-        n_e2e = args.steps
+        n_e2e = steps
         barrier(); torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -407,20 +381,29 @@ def main():
                "overlap": "copies of step i+1 / i-1 run beside the kernels of step i (two buffer slots)"}
 
     if rank != 0:
-        return
+        ctx.close()
+        return None
     # ---- per-kernel table and the roofline of the dominant kernel
     pk, pk_kind = peaks()
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     counts = buf.counts.cpu().numpy()
     work = kernel_work(w, counts)
     kernels = {}
     for name, (tot, calls) in prof.items():
         avg_ms = tot / max(1, calls)
         fl, by = work.get(name, (0, 0))
-        rec = {"ms": round(avg_ms, 4), "launches": calls, "share": round(tot / ms * (1 if world == 1 else 1), 4)}
+        rec = {"ms": round(avg_ms, 4), "launches": calls, "share": round(tot / ms, 4)}
         if fl:
             rec["tflops"] = round(fl / (avg_ms * 1e-3) / 1e12, 1)
         if by:
             rec["gbs"] = round(by / (avg_ms * 1e-3) / 1e9, 1)
+        if fl and by:   # fraction of this kernel's own roofline: the longer of its tensor time and its HBM time
+            t_roof = max(fl / (pk["bf16_tflops_sustained"] * 1e12), by / (pk["hbm_gbs"] * 1e9))
+            rec["roofline_frac"] = round(t_roof / (avg_ms * 1e-3), 3)
+            rec["bound"] = "tensor" if fl / (pk["bf16_tflops_sustained"] * 1e12) >= by / (pk["hbm_gbs"] * 1e9) else "hbm"
+        elif by:
+            rec["roofline_frac"] = round(by / (pk["hbm_gbs"] * 1e9) / (avg_ms * 1e-3), 3)
+            rec["bound"] = "hbm"
         kernels[name] = rec
     roofline = None
     if kernels:
@@ -430,8 +413,8 @@ def main():
         t_tensor = fl / (pk["bf16_tflops_sustained"] * 1e12)
         t_hbm = by / (pk["hbm_gbs"] * 1e9)
         if top == "route_score":
-            # plain fp32 FMA chains: 148 SMs x 128 lanes x 2 flop at the maximum SM clock
-            peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            # plain fp32 FMA chains: SMs x 128 lanes x 2 flop at the maximum SM clock
+            peak = sm_count * 128 * 2 * 1.965e9 / 1e12
             roofline = {"kernel": top, "bound": "alu", "achieved": fl / avg_s / 1e12, "peak": peak, "unit": "TFLOP/s"}
         elif t_tensor >= t_hbm:
             roofline = {"kernel": top, "bound": "tensor", "achieved": fl / avg_s / 1e12,
@@ -446,7 +429,7 @@ def main():
 
     # ---- CPU baseline: the oracle on a bounded sample (complete work of a few experts)
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and with_cpu_baseline:
         import oracle
         oracle.build()
         order = np.argsort(-counts)
@@ -460,21 +443,81 @@ def main():
                "seconds": round(s1 + s2, 2),
                "sample": f"{1 + len(more)} median-load experts, {r1 + r2} rows: "
                          f"{'fwd+dgrad+wgrad' if w.backward else 'fwd'} of every row routed to them"}
-
-    out = {
-        "metric": "moe_layer_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+    ctx.close()
+    return {
+        "metric": "moe_layer_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "T": w.T, "d": w.d, "E": w.E, "k": w.k, "f": w.f,
-                   "pass": "fwd+bwd" if w.backward else "fwd", "l2": "inputs larger than L2",
-                   "load_cv": float(counts.std() / max(1e-9, counts.mean())),
-                   "empty_experts": int((counts == 0).sum())},
+        "config": config_of(w),
+        "routing": {"load_cv": float(counts.std() / max(1e-9, counts.mean())), "empty_experts": int((counts == 0).sum()),
+                    "rows_min": int(counts.min()), "rows_max": int(counts.max())},
         "frac_of_bf16_peak_nominal": value / world / 2250.0,
         "frac_of_bf16_peak_measured": value / world / pk["bf16_tflops_sustained"],
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
         "cpu_baseline": cpu,
     }
-    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=None, choices=sorted(synth.WORKLOADS) + ["vocab_loss", "vocab_train"],
+                    help="default: c5_train as the headline, followed by the forward workloads c2_mid, c3_trillion, "
+                         "c4_skew as sub-records of the same JSON line")
+    ap.add_argument("--shape", default=None,
+                    help="T,d,E,k,f overriding the named workload's sizes (same distributions): small cases for "
+                         "profiler captures")
+    ap.add_argument("--gemm-path", type=int, default=0, help="mop_gemm_path (0 = library default)")
+    ap.add_argument("--with-router-bwd", action="store_true",
+                    help="also run the router backward (dgate -> dW_r, dX) in every step of a fwd+bwd workload")
+    ap.add_argument("--gather", action="store_true",
+                    help="forward-only workloads: up-projection gathers its rows from x (no permuted copy)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra-workloads", action="store_true",
+                    help="default invocation: skip the forward workloads that follow the headline")
+    args = ap.parse_args()
+    extra = args.workload is None and args.shape is None and not args.no_extra_workloads and args.impl == "ours"
+    args.workload = args.workload or "c5_train"
+    if args.workload in ("vocab_loss", "vocab_train"):
+        return run_vocab(args)
+    w = synth.WORKLOADS[args.workload]
+    if args.shape:
+        T, d, E, k, f = (int(v) for v in args.shape.split(","))
+        import dataclasses
+        w = dataclasses.replace(w, T=T, d=d, E=E, k=k, f=f, name=f"{w.name}[{args.shape}]")
+    if args.impl == "reference":
+        args.steps = args.steps or 3
+        args.warmup = 1 if args.warmup is None else args.warmup
+        return run_reference(args, w)
+    args.steps = args.steps or 20
+    args.warmup = max(3, args.warmup or 3)
+
+    rank, local, world = launch.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local)
+    launch.init("nccl", torch.device("cuda", local))
+
+    out = bench_workload(w, args, args.steps, args.warmup, not args.no_cpu_baseline)
+    if extra:
+        # The tensor-bound forward configurations, one after the other on the freed GPU: sub-records of the
+        # same line (metric, config and value of the line stay those of the training configuration).
+        subs = {}
+        for name in ("c2_mid", "c3_trillion", "c4_skew"):
+            torch.cuda.empty_cache()
+            sub = bench_workload(synth.WORKLOADS[name], args, min(args.steps, 20), 3, False)
+            if sub is not None:
+                subs[name] = {k: sub[k] for k in ("ms_per_step", "value", "unit", "steps", "config", "routing", "clocks", "e2e",
+                                                  "gpu_launches", "roofline", "kernels",
+                                                  "frac_of_bf16_peak_nominal", "frac_of_bf16_peak_measured")}
+        if out is not None:
+            out["workloads"] = subs
+    if out is not None:
+        print(json.dumps(out))
 
 
 if __name__ == "__main__":

@@ -310,7 +310,10 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
             const int buf = it & 1;
             const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
-            if (!mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane)) break;
+            bool ready = mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane);
+            // the gate warp and its up warp meet at a named barrier below: they give up together or not at all
+            if constexpr (KIND == TN_F1 || KIND == TN_F1G) ready = bar_vote_all(1 + (quarter & 1), 64, ready);
+            if (!ready) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * 256;
             float v[32];
