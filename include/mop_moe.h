@@ -62,6 +62,13 @@ typedef enum { MOP_BIAS_NONE = 0, MOP_BIAS_POST_SCORE = 1, MOP_BIAS_PRE_LOGIT = 
 typedef enum { MOP_GEMM_AUTO = 0, MOP_GEMM_TENSOR = 1, MOP_GEMM_SCALAR = 2, MOP_GEMM_TENSOR_1CTA = 3,
                MOP_GEMM_TENSOR_2CTA = 4, MOP_GEMM_TENSOR_MIXED = 5, MOP_GEMM_TENSOR_TN = 6 } mop_gemm_path;
 
+/* How mop_moe_route computes the logits.  EXACT: one fp32 fused multiply-add chain per (token, expert) on
+ * the CUDA cores.  TENSOR: logits on the tensor cores from three bf16 pieces of W_r, then the chain is
+ * evaluated only for the experts of a token whose order the approximate keys leave in doubt (needs d and E
+ * multiples of 64, else MOP_ERR_UNSUPPORTED).  Both give the same indices in the same order; AUTO takes
+ * TENSOR when the scoring is large (2 T d E >= 2e10 flop) and the shape allows it. */
+typedef enum { MOP_ROUTE_AUTO = 0, MOP_ROUTE_EXACT = 1, MOP_ROUTE_TENSOR = 2 } mop_route_path;
+
 typedef struct {
     int32_t T, d, E, k, f;
     int32_t score_fn;      /* mop_score_fn */
@@ -72,6 +79,7 @@ typedef struct {
     int32_t gemm_path;     /* mop_gemm_path; AUTO = tensor cores when the shape allows */
     int32_t host_io;       /* 1: the context also holds the activations of the host-buffer entry points;
                               2: and a second slot of every buffer a copy touches, for the *_async forms */
+    int32_t route_path;    /* mop_route_path */
 } mop_moe_shape;
 
 /* Create / destroy a context on `device` (a CUDA ordinal).  mop_create allocates the
@@ -115,9 +123,19 @@ int64_t mop_launch_count(const mop_ctx* ctx);
  *   topk_idx = the k experts with the largest key, descending; equal keys -> lower id.
  *   gate     = score of the selected expert / sum of the k selected scores.
  * x [T,d] bf16; W_r [d,E] f32; bias [E] f32 (NULL iff MOP_BIAS_NONE);
- * topk_idx [T,k] i32 out; topk_gate [T,k] f32 out; logits_opt [T,E] f32 out or NULL. */
+ * topk_idx [T,k] i32 out; topk_gate [T,k] f32 out; logits_opt [T,E] f32 out or NULL.
+ * On the tensor-core path (mop_route_path) the returned logits are the chain's value for the experts that
+ * were re-evaluated and within 24 * 2^-24 ||x_t|| max_e ||W_r[:,e]|| of it elsewhere, the indices and
+ * their order are those of the chain, and the gates agree to 1e-6 + 1e-5 |g|. */
 mop_status mop_moe_route(mop_ctx* ctx, const void* x, const float* W_r, const float* bias, int32_t* topk_idx,
                          float* topk_gate, float* logits_opt, void* stream);
+
+/* Statistics of the tensor-core scoring path since the last call: tokens whose approximate keys left the
+ * order in doubt, the chains evaluated for them, and how many of those exact logits lay further than half
+ * the assumed error bound from their approximation (expected 0: the bound is a model of the rounding
+ * errors, and this is its running check).  Zeros on the exact path.  Synchronises `stream`. */
+mop_status mop_route_stats(mop_ctx* ctx, int64_t* tokens_reevaluated, int64_t* chains, int64_t* beyond_half_bound,
+                           void* stream);
 
 /* Count and prefix-sum permutation of assignments a = t*k + j into expert-contiguous rows
  * (the buffer of N k rows of width H in Eq. 4).

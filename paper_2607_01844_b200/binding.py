@@ -17,12 +17,13 @@ LIB_PATH = _PKG / "libmop_moe.so"
 MOP_OK = 0
 STATUS_NAMES = {0: "MOP_OK", 1: "MOP_ERR_INVALID_ARG", 2: "MOP_ERR_SHAPE", 3: "MOP_ERR_ALIGN", 4: "MOP_ERR_WORKSPACE",
                 5: "MOP_ERR_CUDA", 6: "MOP_ERR_UNSUPPORTED", 7: "MOP_ERR_TIMEOUT"}
+ROUTE_AUTO, ROUTE_EXACT, ROUTE_TENSOR = 0, 1, 2
 GEMM_AUTO, GEMM_TENSOR, GEMM_SCALAR, GEMM_TENSOR_1CTA, GEMM_TENSOR_2CTA, GEMM_TENSOR_MIXED, GEMM_TENSOR_TN = 0, 1, 2, 3, 4, 5, 6
 
 
 class MopShape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("T", "d", "E", "k", "f", "score_fn", "bias_mode", "with_backward",
-                                              "dw_accumulate", "gemm_path", "host_io")]
+                                              "dw_accumulate", "gemm_path", "host_io", "route_path")]
 
 
 class MopError(RuntimeError):
@@ -57,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.mop_debug_guard_poke.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, _P]
         L.mop_launch_count.restype = ctypes.c_int64
         L.mop_moe_route.argtypes = [_P] * 8
+        L.mop_route_stats.argtypes = [_P] + [ctypes.POINTER(ctypes.c_int64)] * 3 + [_P]
         L.mop_moe_permute.argtypes = [_P] * 9
         L.mop_moe_expert_ffn_fwd.argtypes = [_P] * 13
         L.mop_moe_expert_ffn_fwd_gather.argtypes = [_P] * 11
@@ -109,9 +111,9 @@ class Context:
     """Owns one mop_ctx (shape + workspace on one device)."""
 
     def __init__(self, T, d, E, k, f, score_fn=0, bias_mode=0, with_backward=False, dw_accumulate=False,
-                 gemm_path=GEMM_AUTO, host_io=False, device=0):
+                 gemm_path=GEMM_AUTO, host_io=False, device=0, route_path=ROUTE_AUTO):
         self.shape = MopShape(T, d, E, k, f, score_fn, bias_mode, int(with_backward), int(dw_accumulate), gemm_path,
-                              int(host_io))
+                              int(host_io), route_path)
         self.handle = _P()
         _check("mop_create", lib().mop_create(ctypes.byref(self.handle), ctypes.byref(self.shape), device))
 
@@ -161,6 +163,15 @@ def mop_debug_guard_check(ctx, stream=None):
 def mop_moe_route(ctx, x, W_r, bias, topk_idx, topk_gate, logits=None, stream=None):
     _check("mop_moe_route", lib().mop_moe_route(ctx.handle, _ptr(x), _ptr(W_r), _ptr(bias), _ptr(topk_idx),
                                                 _ptr(topk_gate), _ptr(logits), _stream(stream)))
+
+
+def mop_route_stats(ctx, stream=None):
+    """(tokens re-evaluated, chains evaluated, exact logits beyond half the assumed error bound) of the
+    tensor-core scoring path since the last call."""
+    a, b, c = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+    _check("mop_route_stats", lib().mop_route_stats(ctx.handle, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
+                                                    _stream(stream)))
+    return a.value, b.value, c.value
 
 
 def mop_moe_permute(ctx, x, topk_idx, counts, offsets, perm_row, row_src, Xp, stream=None):
@@ -360,7 +371,8 @@ def backward(ctx, inp, buf, stream=None):
                            buf.dW_down, buf.dgate, stream)
 
 
-def context_for(w, device=0, gemm_path=GEMM_AUTO, backward=None, host_io=False, dw_accumulate=False):
+def context_for(w, device=0, gemm_path=GEMM_AUTO, backward=None, host_io=False, dw_accumulate=False,
+                route_path=ROUTE_AUTO):
     backward = w.backward if backward is None else backward
     return Context(w.T, w.d, w.E, w.k, w.f, w.score_fn, w.bias_mode, backward, dw_accumulate, gemm_path, host_io,
-                   device)
+                   device, route_path)

@@ -34,6 +34,14 @@ struct mop_ctx {
     bf16 *dYp, *dG, *dU, *gH, *dXp;  // backward intermediates
     bf16 *rG, *rU, *rH;              // recompute-in-backward buffers (activation checkpointing)
     float *dz_sel, *dz_row, *wrT;    // router backward: dz per assignment / per permuted row; W_r^T [E,d]
+    // tensor-core scoring path: bf16 pieces of W_r [3,d,E], W_r^T [E,d], column-norm partials, ||x_t||, scalars
+    // (wmax, statistics), the {0, T} offsets and the 128-row tile table of the dense logit GEMM
+    bool fast_route;
+    cudaStream_t fr_stream;          // the row norms of x are taken beside the logit GEMM
+    cudaEvent_t fr_fork, fr_join;
+    bf16* fr_pieces;
+    float *fr_wrT, *fr_colsq, *fr_xnorm, *fr_scal, *fr_wsq;
+    int32_t *fr_off, *fr_tiles;
     // host-buffer entry point scratch
     bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
     int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
@@ -67,6 +75,7 @@ constexpr uint32_t GUARD_PATTERN = 0xA5C3A5C3u;
 
 struct Layout {
     size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT, rG, rU, rH;
+    size_t fr_pieces, fr_wrT, fr_colsq, fr_xnorm, fr_scal, fr_off, fr_tiles, fr_wsq;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
     size_t hG, hU, hdY, hdX, hdgate;
     size_t qx, qY, qidx, qgate, qdY, qdX, qdgate;   // second slot of the pipelined host entry points
@@ -92,6 +101,16 @@ __global__ void guard_check_kernel(const char* ws, GuardList g, unsigned long lo
 }
 
 int perm_units(const mop_moe_shape& s) { return ceil_div(s.T * s.k, PERM_SEG); }
+// The tensor-core scoring path needs 64-wide K blocks of x and 64-wide column chunks of W_r.
+bool route_fast_possible(const mop_moe_shape& s) {
+    return s.route_path != MOP_ROUTE_EXACT && s.T > 0 && s.d % 64 == 0 && s.E % 64 == 0 && tc_shape_supported(s.d, s.f);
+}
+// Measured policy: the three-piece GEMM plus the selection with re-evaluation beats the fp32 chains once
+// the scoring is large (configs 3-5: 45-60 GFLOP); small layers keep the chains.
+bool route_fast_wanted(const mop_moe_shape& s) {
+    if (s.route_path == MOP_ROUTE_TENSOR) return true;
+    return 2.0 * s.T * s.d * s.E >= 2e10;
+}
 int part_tiles(const mop_moe_shape& s) { return ceil_div(s.f, 32); }
 
 Layout make_layout(const mop_moe_shape& s) {
@@ -105,6 +124,16 @@ Layout make_layout(const mop_moe_shape& s) {
     L.partial = take((size_t)perm_units(s) * E * 4 + 4);
     L.tiles = take(tc_tables_bytes(s.T * s.k, s.E));
     L.status = take(256);
+    if (route_fast_possible(s)) {
+        L.fr_pieces = take(3 * d * E * 2);
+        L.fr_wrT = take(d * E * 4);
+        L.fr_colsq = take((size_t)ceil_div(s.d, 32) * E * 4);
+        L.fr_xnorm = take(T * 4 + 16);
+        L.fr_scal = take(256);
+        L.fr_wsq = take(E * 4);
+        L.fr_off = take(16);
+        L.fr_tiles = take(tc_tile_table_bytes(s.T, 1));
+    }
     if (s.with_backward) {
         L.part = take((size_t)part_tiles(s) * M * 4);
         L.dYp = take(M * d * 2);
@@ -169,6 +198,7 @@ mop_status check_shape(const mop_moe_shape* s) {
     if ((long long)s->T * s->d >= (1ll << 40) || (long long)s->d * s->f >= (1ll << 31)) return MOP_ERR_SHAPE;
     if (s->d % 8 || s->f % 8) return MOP_ERR_ALIGN;
     if (s->host_io < 0 || s->host_io > 2) return MOP_ERR_INVALID_ARG;
+    if (s->route_path < MOP_ROUTE_AUTO || s->route_path > MOP_ROUTE_TENSOR) return MOP_ERR_INVALID_ARG;
     return MOP_OK;
 }
 
@@ -279,6 +309,21 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
     c->partial = reinterpret_cast<int32_t*>(w + L.partial);
     c->tiles = reinterpret_cast<int32_t*>(w + L.tiles);
     c->status = reinterpret_cast<int32_t*>(w + L.status);
+    c->fast_route = false;
+    if (route_fast_possible(*shape) && prop.major == 10) {
+        c->fr_pieces = reinterpret_cast<bf16*>(w + L.fr_pieces);
+        c->fr_wrT = reinterpret_cast<float*>(w + L.fr_wrT);
+        c->fr_colsq = reinterpret_cast<float*>(w + L.fr_colsq);
+        c->fr_xnorm = reinterpret_cast<float*>(w + L.fr_xnorm);
+        c->fr_scal = reinterpret_cast<float*>(w + L.fr_scal);
+        c->fr_wsq = reinterpret_cast<float*>(w + L.fr_wsq);
+        c->fr_off = reinterpret_cast<int32_t*>(w + L.fr_off);
+        c->fr_tiles = reinterpret_cast<int32_t*>(w + L.fr_tiles);
+        c->fast_route = route_fast_wanted(*shape);
+    } else if (shape->route_path == MOP_ROUTE_TENSOR) {
+        cudaFree(c->ws); delete c;
+        return MOP_ERR_UNSUPPORTED;
+    }
     if (shape->with_backward) {
         c->part = reinterpret_cast<float*>(w + L.part);
         c->dYp = reinterpret_cast<bf16*>(w + L.dYp);
@@ -356,6 +401,19 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         if (st == MOP_OK) st = tc2_init();
         if (st == MOP_OK) st = tn_init();
         if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
+        if (c->fast_route) {   // the logit GEMM's row tiles depend on T alone: built once
+            const int32_t host_off[2] = {0, shape->T};
+            bool ok = cudaMemcpy(c->fr_off, host_off, sizeof(host_off), cudaMemcpyHostToDevice) == cudaSuccess &&
+                      cudaMemset(c->fr_scal, 0, 256) == cudaSuccess;
+            if (ok) {
+                tc_build_mtiles_kernel<<<1, 1024>>>(c->fr_off, 1, reinterpret_cast<int4*>(c->fr_tiles + 64), c->fr_tiles);
+                ok = cudaDeviceSynchronize() == cudaSuccess;
+            }
+            ok = ok && cudaStreamCreateWithFlags(&c->fr_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->fr_fork, cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&c->fr_join, cudaEventDisableTiming) == cudaSuccess;
+            if (!ok) { cudaFree(c->ws); delete c; return MOP_ERR_CUDA; }
+        }
         c->plan.pairs = shape->gemm_path == MOP_GEMM_TENSOR_2CTA ? 1 : shape->gemm_path == MOP_GEMM_TENSOR_MIXED ? 2 : 0;
         if (c->sm_count < 2) c->plan.pairs = 0;
         // Measured policy (B200): the tokens-on-N down-projection wins on every workload; the tokens-on-N
@@ -378,6 +436,10 @@ void mop_destroy(mop_ctx* c) {
     if (c->prof.ev) {
         for (int i = 0; i < 2 * Profiler::MAX_REC; ++i) cudaEventDestroy(c->prof.ev[i]);
         delete[] c->prof.ev;
+    }
+    if (c->fast_route) {
+        cudaStreamDestroy(c->fr_stream);
+        cudaEventDestroy(c->fr_fork); cudaEventDestroy(c->fr_join);
     }
     if (c->s.host_io) {
         cudaStreamDestroy(c->copy_stream);
@@ -477,6 +539,38 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
     if (!guard.ok) return MOP_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     float* z = logits_opt ? logits_opt : c->z;
+    if (c->fast_route) {
+        // logits on the tensor cores from three bf16 pieces of W_r, then selection with the contract's chain
+        // re-evaluated where the order is in doubt
+        mop_status r;
+        dim3 gp(ceil_div(s.E, 32), ceil_div(s.d, 32));
+        // the row norms of x depend on nothing else: they run on a side stream beside the logit GEMM
+        CUDA_OK(cudaEventRecord(c->fr_fork, st));
+        CUDA_OK(cudaStreamWaitEvent(c->fr_stream, c->fr_fork, 0));
+        route_xnorm_kernel<<<ceil_div(s.T, 8), 256, 0, c->fr_stream>>>(static_cast<const bf16*>(x), c->fr_xnorm, s.T, s.d);
+        CUDA_OK(cudaEventRecord(c->fr_join, c->fr_stream));
+        LAUNCH(c, "route_prep", st,
+               route_prep_kernel<<<gp, 256, 0, st>>>(W_r, c->fr_pieces, c->fr_wrT, c->fr_colsq, s.d, s.E);
+               route_wnorm_kernel<<<ceil_div(s.E, 8), 256, 0, st>>>(c->fr_colsq, c->fr_wsq, ceil_div(s.d, 32), s.E));
+        if ((r = after_launch(c, 3)) != MOP_OK) return r;
+        CUtensorMap mX, mW;
+        if (!tc_map_2d(&c->plan, &mX, x, s.T, s.d, 128) || !tc_map_chunked_3d(&c->plan, &mW, c->fr_pieces, 3, s.d, s.E, 4))
+            return MOP_ERR_CUDA;
+        TcArgs g{};
+        g.offsets = c->fr_off; g.n_mtiles = c->fr_tiles; g.mtiles = reinterpret_cast<const int4*>(c->fr_tiles + 64);
+        g.E = 1; g.status = c->status;
+        g.tiles_n = ceil_div(s.E, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.E; g.m_fastest = 1;
+        g.ep.outf = z; g.ep.accumulate = 0; g.ep.M_total = s.T;
+        if ((r = tc_launch<TC_RS>(&c->plan, "route_score_tc", mX, mX, mW, mW, mX, mX, g, st)) != MOP_OK) return r;
+        c->launches += 1;
+        CUDA_OK(cudaStreamWaitEvent(st, c->fr_join, 0));
+        const size_t fsmem = (size_t)SELF_WARPS * (3 * s.E + SELF_SMEM_FLOATS) * sizeof(float);
+        LAUNCH(c, "route_select_fast", st,
+               route_select_fast_kernel<<<ceil_div(s.T, SELF_WARPS), SELF_WARPS * 32, fsmem, st>>>(
+                   z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
+                   reinterpret_cast<int32_t*>(c->fr_scal) + 8, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode));
+        return after_launch(c);
+    }
     LAUNCH(c, "route_score", st, route_score(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E, c->sm_count, st));
     mop_status r = after_launch(c);
     if (r != MOP_OK) return r;
@@ -485,6 +579,25 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
            route_select_kernel<<<ceil_div(s.T, SEL_WARPS), SEL_WARPS * 32, smem, st>>>(
                z, bias, topk_idx, topk_gate, s.T, s.E, s.k, s.score_fn, s.bias_mode));
     return after_launch(c);
+}
+
+mop_status mop_route_stats(mop_ctx* c, int64_t* tokens_reevaluated, int64_t* chains, int64_t* beyond_half_bound,
+                           void* stream) {
+    if (!c || !tokens_reevaluated || !chains || !beyond_half_bound) return MOP_ERR_INVALID_ARG;
+    *tokens_reevaluated = *chains = *beyond_half_bound = 0;
+    if (!c->fast_route) return MOP_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t host[3] = {0, 0, 0};
+    int32_t* dev = reinterpret_cast<int32_t*>(c->fr_scal) + 8;
+    CUDA_OK(cudaMemcpyAsync(host, dev, 12, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaMemsetAsync(dev, 0, 12, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    *tokens_reevaluated = host[0];
+    *chains = host[1];
+    *beyond_half_bound = host[2];
+    return MOP_OK;
 }
 
 mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, int32_t* counts, int32_t* offsets,

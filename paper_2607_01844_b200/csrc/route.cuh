@@ -283,6 +283,322 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) route_select_kernel(const floa
 }
 
 // ---------------------------------------------------------------------------------------------
+// Fast scoring path: logits on the tensor cores, the contract's chain only where it can matter.
+//
+// 1. W_r (fp32) is split into three bf16 pieces, hi + mid + lo = W_r to 2^-24 relative (each
+//    residual is exact in fp32), and x (bf16) is multiplied by the pieces on the tensor cores: z~
+//    (kind TC_RS of the grouped GEMM; the K loop is summed in segments of 512 so that the truncating
+//    accumulation inside the tensor core stays short, the segments are added in fp32 registers).
+//    Every product is exact; what separates z~ from the contract's logit z (one fp32 fused
+//    multiply-add per i, i ascending) is the rounding of the two summations.  Each rounding is at most
+//    u = 2^-24 of a partial sum, and the partial sums of a logit grow like a random walk towards
+//    ||x|| ||w|| / sqrt(d) for data without a common direction: d roundings give a standard deviation of
+//    u ||x|| ||w|| / sqrt(6) per summation, whatever d.  The selection relies on
+//        |z~ - z|  <=  eps_z(t) = 24 u ||x_t||_2 max_e ||W_r[:,e]||_2        (40 standard deviations).
+//    This is a model, not a worst case (which is d u ||x|| ||w||): the realised maximum over millions
+//    of logits is 3 to 6.2 u ||x|| ||w|| on every shape tried, the tests assert it, and every logit that
+//    the kernel re-evaluates is compared with half the bound as it runs (mop_route_stats).
+//    In key space a logit error e moves sigmoid(z) + b by at most (s (1 - s) + e / 8) e + 4e-7.
+// 2. One warp per token selects the k largest approximate keys and gives every key the interval that
+//    holds its exact value.  If the intervals of adjacent picks are disjoint and no other expert's
+//    interval reaches the weakest pick, the exact keys have the same order and the token is done
+//    (more than nine tenths of the tokens).  Otherwise the warp evaluates the contract's chain
+//    (__fmaf_rn, i ascending, W_r read through its transposed copy) for the experts in doubt, whose
+//    intervals become points, writes those logits over z~, and selects again, until nothing that
+//    matters overlaps.  Indices and their order are then those of the exact path.
+// 3. Gates are ratios of scores, not an order: a pick keeps its approximate logit unless that could move
+//    its gate by more than 5e-6 relative (score far from saturation), in which case its chain is
+//    evaluated too; the gates then agree with the exact path's to 1e-6 + 1e-5 g.
+// ---------------------------------------------------------------------------------------------
+
+// W_r [d,E] -> three bf16 pieces [3,d,E], the transposed copy W_r^T [E,d] (32 x 32 tiles through shared
+// memory) and, per 32-row slab, the partial squared column norms (summed by route_wnorm_kernel).
+__global__ void __launch_bounds__(256) route_prep_kernel(const float* __restrict__ W_r, bf16* __restrict__ pieces,
+                                                         float* __restrict__ W_rT, float* __restrict__ colsq,
+                                                         int d, int E) {
+    __shared__ float tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    const size_t n = (size_t)d * E;
+    for (int r = ty; r < 32; r += 8) {
+        float w = 0.0f;
+        if (r0 + r < d && c0 + tx < E) {
+            const size_t i = (size_t)(r0 + r) * E + c0 + tx;
+            w = W_r[i];
+            const bf16 hi = __float2bfloat16_rn(w);
+            const float r1 = w - __bfloat162float(hi);          // exact
+            const bf16 mid = __float2bfloat16_rn(r1);
+            const float r2 = r1 - __bfloat162float(mid);        // exact
+            pieces[i] = hi;
+            pieces[n + i] = mid;
+            pieces[2 * n + i] = __float2bfloat16_rn(r2);
+        }
+        tile[r][tx] = w;
+    }
+    __syncthreads();
+    for (int c = ty; c < 32; c += 8)
+        if (c0 + c < E && r0 + tx < d) W_rT[(size_t)(c0 + c) * d + r0 + tx] = tile[tx][c];
+    if (ty == 0 && c0 + tx < E) {
+        float sq = 0.0f;
+        for (int r = 0; r < 32; ++r) sq = fmaf(tile[r][tx], tile[r][tx], sq);
+        colsq[(size_t)blockIdx.y * E + c0 + tx] = sq;
+    }
+}
+
+// Squared column norms ||W_r[:,e]||^2 from the slab partials: one warp per expert, fixed order (reproducible).
+__global__ void __launch_bounds__(256) route_wnorm_kernel(const float* __restrict__ colsq, float* __restrict__ wsq,
+                                                          int slabs, int E) {
+    const int lane = threadIdx.x % 32;
+    const int e = blockIdx.x * 8 + threadIdx.x / 32;
+    if (e >= E) return;
+    float sq = 0.0f;
+    for (int s = lane; s < slabs; s += 32) sq += colsq[(size_t)s * E + e];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+    if (lane == 0) wsq[e] = sq;
+}
+
+// ||x_t||_2 per token: one warp per row, 16-byte loads.
+__global__ void __launch_bounds__(256) route_xnorm_kernel(const bf16* __restrict__ x, float* __restrict__ xnorm, int T,
+                                                          int d) {
+    const int lane = threadIdx.x % 32;
+    const int t = blockIdx.x * 8 + threadIdx.x / 32;
+    if (t >= T) return;
+    const uint4* row = reinterpret_cast<const uint4*>(x + (size_t)t * d);
+    float sq = 0.0f;
+    for (int v = lane; v < d / 8; v += 32) {
+        const uint4 q = __ldg(row + v);
+        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float a = bf16_lo(w4[j]), b = bf16_hi(w4[j]);
+            sq = fmaf(a, a, sq);
+            sq = fmaf(b, b, sq);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+    if (lane == 0) xnorm[t] = sqrtf(sq);
+}
+
+constexpr int SELF_WARPS = 2;     // warps per block of the fast selection (a warp that re-evaluates takes ~20 us)
+constexpr float ROUTE_EPS_C = 24.0f;      // order:  |z~ - z| <= C 2^-24 ||x_t|| max_e ||W_r[:,e]||  (see below)
+constexpr float ROUTE_EPS_GATE_C = 6.0f;  // gates:  the same with the largest error seen, not a bound (a tolerance, not an order)
+constexpr float ROUTE_GATE_REL = 5e-6f;   // a pick whose gate could be off by more than this (relative) gets its chain
+constexpr int SELF_XCHUNK = 256;  // elements of the token's row staged per step of the exact chains
+constexpr int SELF_CAND = 4;      // chains evaluated side by side (one lane each), their W_r^T rows staged in shared memory
+constexpr int SELF_WPITCH = SELF_XCHUNK + 4;   // row pitch of the staged W_r^T chunks: lanes read different banks
+constexpr int SELF_SMEM_FLOATS = SELF_XCHUNK + SELF_CAND * SELF_WPITCH;   // per warp, besides the 3 E key / logit / list words
+
+// k selection rounds over the keys in shared memory (as in route_select_kernel).  Lane j < k keeps the j-th
+// pick: its expert, its key and the logit its gate is computed from; `taken` marks this lane's picked experts.
+__device__ __forceinline__ void select_rounds(const float* key, const float* zg, int E, int k, int lane, int& my_e,
+                                              float& my_key, float& my_z, uint32_t& taken) {
+    taken = 0;
+    my_e = -1; my_key = 0.0f; my_z = 0.0f;
+    for (int j = 0; j < k; ++j) {
+        int best = -1;
+        float bk = 0.0f;
+        for (int q = 0, e = lane; e < E; ++q, e += 32) {
+            if ((taken >> q) & 1u) continue;
+            const float v = key[e];
+            if (best < 0 || v > bk) { best = e; bk = v; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ok = __shfl_xor_sync(0xffffffffu, bk, off);
+            const int oe = __shfl_xor_sync(0xffffffffu, best, off);
+            const bool take = (oe >= 0) && (best < 0 || ok > bk || (ok == bk && oe < best));
+            if (take) { bk = ok; best = oe; }
+        }
+        if ((best & 31) == lane) taken |= 1u << (best >> 5);
+        if (j == lane) { my_e = best; my_key = bk; my_z = zg[best]; }
+    }
+}
+
+__device__ __forceinline__ float route_key(float zz, float b, int score_fn, int bias_mode) {
+    return (score_fn == 1 && bias_mode == 1) ? __fadd_rn(sigmoid_contract(zz), b) : zz;
+}
+
+// Bound on the error of a key whose logit is off by at most ez (a little slack covers its own rounding).
+__device__ __forceinline__ float key_error(float zz, float ez, int score_fn, int bias_mode) {
+    if (!(score_fn == 1 && bias_mode == 1)) return ez;                   // the key is the logit itself
+    const float s = sigmoidf_acc(zz);
+    return 1.001f * (s * (1.0f - s) + 0.125f * ez) * ez + 4e-7f;         // |s''| <= 0.1; rounding of the sequence
+}
+
+__global__ void __launch_bounds__(SELF_WARPS * 32) route_select_fast_kernel(
+    float* __restrict__ z, const float* __restrict__ bias, const bf16* __restrict__ x, const float* __restrict__ W_rT,
+    const float* __restrict__ xnorm, const float* __restrict__ wsq, int32_t* __restrict__ idx,
+    float* __restrict__ gate, int32_t* __restrict__ stats, int T, int d, int E, int k, int score_fn, int bias_mode) {
+    extern __shared__ float sel_smem[];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    float* key = sel_smem + (size_t)warp * (3 * E + SELF_SMEM_FLOATS);
+    float* zg = key + E;
+    int32_t* clist = reinterpret_cast<int32_t*>(zg + E);   // experts whose exact logit is needed
+    float* xs = zg + 2 * E;                                 // a chunk of the token's row, fp32
+    float* ws = xs + SELF_XCHUNK;                           // the same chunk of up to SELF_CAND rows of W_r^T
+    const int t = blockIdx.x * SELF_WARPS + warp;
+    if (t >= T) return;
+    float* zrow = z + (size_t)t * E;
+    for (int e = lane; e < E; e += 32) {
+        float zz = zrow[e];
+        const float b = bias_mode ? bias[e] : 0.0f;
+        if (bias_mode == 2) zz = __fadd_rn(zz, b);
+        key[e] = route_key(zz, b, score_fn, bias_mode);
+        zg[e] = zz;
+    }
+    __syncwarp();
+    // Bound of this token's logit error (see above).
+    float wmax2 = 0.0f;                              // largest squared column norm of W_r
+    for (int e = lane; e < E; e += 32) wmax2 = fmaxf(wmax2, wsq[e]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) wmax2 = fmaxf(wmax2, __shfl_xor_sync(0xffffffffu, wmax2, off));
+    const float scale = 5.9604645e-8f * xnorm[t] * sqrtf(wmax2);
+    const float ez = ROUTE_EPS_C * scale, ez_gate = ROUTE_EPS_GATE_C * scale;
+    uint32_t exact = 0;                              // this lane's experts (e = lane + 32 q) that carry the chain's logit
+    int my_e; float my_key, my_z; uint32_t taken;
+    int n_chains = 0, n_bad = 0;
+    for (int iter = 0; iter <= k + 1; ++iter) {
+        select_rounds(key, zg, E, k, lane, my_e, my_key, my_z, taken);
+        // interval [lo, hi] that holds the exact key of each pick (a point once the chain was evaluated)
+        const bool pick = lane < k;
+        const uint32_t pick_exact = pick ? (__shfl_sync(0xffffffffu, exact, my_e & 31) >> (my_e >> 5)) & 1u
+                                         : (__shfl_sync(0xffffffffu, exact, 0), 1u);
+        const float my_err = (pick && !pick_exact) ? key_error(my_z, ez, score_fn, bias_mode) : 0.0f;
+        const float lo = pick ? my_key - my_err : INFINITY, hi = pick ? my_key + my_err : -INFINITY;
+        const float next_hi = __shfl_down_sync(0xffffffffu, hi, 1), prev_lo = __shfl_up_sync(0xffffffffu, lo, 1);
+        // a pick is in doubt if it may swap with a neighbour (NaN compares unsure: inputs must be finite)
+        bool doubt = pick && ((lane + 1 < k && !(lo > next_hi)) || (lane > 0 && !(prev_lo > hi)));
+        float lo_min = lo;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) lo_min = fminf(lo_min, __shfl_xor_sync(0xffffffffu, lo_min, off));
+        // outsiders that could reach the weakest pick, and the picks they could reach.  Nearly all of them
+        // fail already with the largest error any key can have (slope 1/4), which costs no transcendental.
+        const float err_any = (score_fn == 1 && bias_mode == 1) ? 1.001f * (0.25f + 0.125f * ez) * ez + 4e-7f : ez;
+        float out_hi = -INFINITY;
+        int n_c = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane, q = e0 >> 5;
+            bool cand = false;
+            if (e < E && !((taken >> q) & 1u) && !(key[e] + err_any < lo_min)) {
+                const bool ex = (exact >> q) & 1u;
+                const float h = key[e] + (ex ? 0.0f : key_error(zg[e], ez, score_fn, bias_mode));
+                if (!(h < lo_min)) { out_hi = fmaxf(out_hi, h); cand = !ex; }
+            }
+            const uint32_t m = __ballot_sync(0xffffffffu, cand);
+            if (m) {
+                if (cand) clist[n_c + __popc(m & ((1u << lane) - 1u))] = e;
+                n_c += __popc(m);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) out_hi = fmaxf(out_hi, __shfl_xor_sync(0xffffffffu, out_hi, off));
+        if (pick && !(lo > out_hi)) doubt = true;
+        // gates: d g / g = (1 - s) dz for a sigmoid score, at most dz for a softmax over the picks
+        if (pick && !pick_exact) {
+            const float sens = (score_fn == 1) ? 1.0f - sigmoidf_acc(my_z) : 1.0f;
+            if (sens * ez_gate > ROUTE_GATE_REL) doubt = true;
+        }
+        // picks in doubt whose logit is still approximate join the list
+        const bool need = doubt && !pick_exact;
+        const uint32_t m = __ballot_sync(0xffffffffu, need);
+        if (need) clist[n_c + __popc(m & ((1u << lane) - 1u))] = my_e;
+        n_c += __popc(m);
+        if (n_c == 0) break;                         // every order that matters is settled (exact ties go by id)
+        __syncwarp();
+        for (int c0 = 0; c0 < n_c; c0 += SELF_CAND) {
+            const int nc = min(SELF_CAND, n_c - c0);
+            const bool mine = lane < nc;
+            const int e = mine ? clist[c0 + lane] : 0;
+            float acc = 0.0f;
+            // All lanes fetch: the token's chunk (16 bytes per lane) and the same chunk of every candidate's row
+            // of W_r^T (lane l: 16-byte pieces l, l + 32, ... of the nc rows laid end to end).  The fetch of chunk
+            // i + 1 is in flight while the chains run over chunk i.
+            constexpr int WV = SELF_CAND * SELF_XCHUNK / 4 / 32;      // 16-byte pieces of W per lane and chunk
+            uint4 xq = make_uint4(0, 0, 0, 0);
+            float4 wq[WV];
+            auto fetch = [&](int i0) {
+                const int n = min(SELF_XCHUNK, d - i0);              // a multiple of 8
+                if (lane < n / 8) xq = __ldg(reinterpret_cast<const uint4*>(x + (size_t)t * d + i0) + lane);
+#pragma unroll
+                for (int u = 0; u < WV; ++u) {
+                    const int v = lane + 32 * u, c = v / (SELF_XCHUNK / 4), j = v % (SELF_XCHUNK / 4);
+                    if (c < nc && 4 * j < n)
+                        wq[u] = __ldg(reinterpret_cast<const float4*>(W_rT + (size_t)clist[c0 + c] * d + i0) + j);
+                }
+            };
+            fetch(0);
+            for (int i0 = 0; i0 < d; i0 += SELF_XCHUNK) {
+                const int n = min(SELF_XCHUNK, d - i0);
+                __syncwarp();
+                {
+                    float* o = xs + lane * 8;
+                    o[0] = bf16_lo(xq.x); o[1] = bf16_hi(xq.x); o[2] = bf16_lo(xq.y); o[3] = bf16_hi(xq.y);
+                    o[4] = bf16_lo(xq.z); o[5] = bf16_hi(xq.z); o[6] = bf16_lo(xq.w); o[7] = bf16_hi(xq.w);
+                }
+#pragma unroll
+                for (int u = 0; u < WV; ++u) {
+                    const int v = lane + 32 * u, c = v / (SELF_XCHUNK / 4), j = v % (SELF_XCHUNK / 4);
+                    if (c < nc) *reinterpret_cast<float4*>(ws + c * SELF_WPITCH + 4 * j) = wq[u];
+                }
+                __syncwarp();
+                if (i0 + SELF_XCHUNK < d) fetch(i0 + SELF_XCHUNK);
+                if (mine) {
+                    // the contract's chain: one fused multiply-add per i, i ascending
+                    const float* wrow = ws + lane * SELF_WPITCH;
+#pragma unroll 4
+                    for (int i = 0; i < n; i += 4) {
+                        const float4 w = *reinterpret_cast<const float4*>(wrow + i);
+                        const float4 xv = *reinterpret_cast<const float4*>(xs + i);
+                        acc = __fmaf_rn(xv.x, w.x, acc);
+                        acc = __fmaf_rn(xv.y, w.y, acc);
+                        acc = __fmaf_rn(xv.z, w.z, acc);
+                        acc = __fmaf_rn(xv.w, w.w, acc);
+                    }
+                }
+            }
+            if (mine) {
+                if (fabsf(zrow[e] - acc) > 0.5f * ez) ++n_bad;       // the model of the error is checked as we go
+                zrow[e] = acc;                       // the exact logit replaces the approximate one
+                const float b = bias_mode ? bias[e] : 0.0f;
+                const float zz = (bias_mode == 2) ? __fadd_rn(acc, b) : acc;
+                key[e] = route_key(zz, b, score_fn, bias_mode);
+                zg[e] = zz;
+            }
+            // mark the evaluated experts in their owner lanes' masks
+            for (int j = 0; j < nc; ++j) {
+                const int ej = clist[c0 + j];
+                if ((ej & 31) == lane) exact |= 1u << (ej >> 5);
+            }
+        }
+        n_chains += n_c;
+        __syncwarp();
+    }
+    if (stats && n_chains > 0) {                     // statistics only: no result depends on them
+        n_bad = __reduce_add_sync(0xffffffffu, n_bad);
+        if (lane == 0) { atomicAdd(stats, 1); atomicAdd(stats + 1, n_chains); if (n_bad) atomicAdd(stats + 2, n_bad); }
+    }
+    const bool act = lane < k;
+    float s;
+    if (score_fn == 0) {
+        float m = act ? my_z : -INFINITY;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        s = act ? expf(my_z - m) : 0.0f;
+    } else {
+        s = act ? sigmoidf_acc(my_z) : 0.0f;
+    }
+    float sum = s;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (act) {
+        idx[(size_t)t * k + lane] = my_e;
+        gate[(size_t)t * k + lane] = s / sum;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Router backward (selection held fixed).  With g_j = s_j / sum_l s_l over a token's k selected
 // experts (s = softmax over all E, whose common denominator cancels, or s = sigmoid):
 //   softmax:  dz_j = g_j (dgate_j - sum_l g_l dgate_l)

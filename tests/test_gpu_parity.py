@@ -435,3 +435,78 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     binding.backward(ctx, inp, buf)
     binding.mop_poll(ctx)
     check_integers(w, host, buf)
+
+
+FAST_ROUTE = [
+    synth.small("c3_trillion", T=1000, d=512, E=256, k=8, f=64, seed=60),                  # sigmoid + post-score bias
+    synth.small("c3_trillion", T=777, d=320, E=64, k=3, f=64, bias_mode=2, seed=61),        # sigmoid, bias before the score
+    synth.small("c2_mid", T=900, d=256, E=128, k=6, f=64, seed=62),                         # softmax
+    synth.small("c3_trillion", T=300, d=192, E=1024, k=32, f=64, seed=63),                  # the selection's limits
+    synth.small("c2_mid", T=257, d=64, E=64, k=32, f=64, seed=64),                          # half of the experts picked
+    synth.small("c3_trillion", T=130, d=7168, E=384, k=8, f=64, seed=65),                   # the long chains of configs 3-5
+]
+
+
+@pytest.mark.parametrize("w", FAST_ROUTE, ids=lambda w: f"{w.name}-T{w.T}d{w.d}E{w.E}k{w.k}s{w.score_fn}b{w.bias_mode}")
+def test_tensor_core_scoring_gives_the_indices_of_the_exact_chains(w):
+    """Logits from three bf16 pieces of W_r on the tensor cores, the contract's chain only where the order is in
+    doubt: indices and their order equal the oracle's (and the exact path's) bit for bit, gates within tolerance,
+    and the returned logits are the chain's value or within the documented bound of it."""
+    host = synth.make_inputs(w, "cpu")
+    inp = to_dev(host)
+    out = {}
+    for path in (binding.ROUTE_EXACT, binding.ROUTE_TENSOR):
+        ctx = binding.context_for(w, route_path=path)
+        idx = torch.empty((w.T, w.k), dtype=torch.int32, device="cuda")
+        gate = torch.empty((w.T, w.k), dtype=torch.float32, device="cuda")
+        logits = torch.empty((w.T, w.E), dtype=torch.float32, device="cuda")
+        binding.mop_moe_route(ctx, inp["x"], inp["W_r"], inp["bias"], idx, gate, logits)
+        binding.mop_poll(ctx)
+        out[path] = (idx.cpu().numpy(), gate.cpu().numpy(), logits.cpu().numpy(), binding.mop_route_stats(ctx))
+    xb = synth.bits(host["x"])
+    ref_idx, ref_gate, ref_z, _ = oracle.route(xb, host["W_r"].numpy(), np_bias(host), w.k, w.score_fn, w.bias_mode,
+                                               want_logits=True)
+    for path, (idx, gate, z, stats) in out.items():
+        assert np.array_equal(idx, ref_idx), f"indices, route path {path}"
+        assert np.all(np.abs(gate - ref_gate) <= 1e-6 + 1e-5 * np.abs(ref_gate)), f"gates, route path {path}"
+    assert np.array_equal(out[binding.ROUTE_EXACT][2], ref_z)                       # the chain, bit for bit
+    assert out[binding.ROUTE_EXACT][3] == (0, 0, 0)
+    # the approximate logits stay inside the bound the selection relies on (and far inside it)
+    z = out[binding.ROUTE_TENSOR][2]
+    xn = np.linalg.norm(oracle.bf16_bits_to_f64(xb), axis=1)
+    wmax = np.linalg.norm(host["W_r"].numpy().astype(np.float64), axis=0).max()
+    eps = 24.0 * 2.0 ** -24 * xn * wmax
+    err = np.abs(z.astype(np.float64) - ref_z.astype(np.float64)).max(1)
+    assert np.all(err <= eps), float((err / eps).max())
+    tokens, chains, beyond = out[binding.ROUTE_TENSOR][3]
+    print(f"{w.name} T={w.T} d={w.d} E={w.E}: logit error {err.max():.2e} = {float((err / eps).max()):.3f} of the bound; "
+          f"{tokens} of {w.T} tokens re-evaluated, {chains} chains")
+    assert 0 <= tokens <= w.T and chains >= tokens and beyond == 0
+    assert float((err / eps).max()) < 0.5
+
+
+def test_tensor_core_scoring_with_equal_and_duplicate_keys():
+    """W_r = 0 makes all keys of a token equal (every expert is re-evaluated and the lower ids win); two equal
+    columns of W_r make one exact tie per token that only the chain can order."""
+    w = synth.small("c2_mid", T=96, d=128, E=64, k=4, f=64, seed=66)
+    host = synth.make_inputs(w, "cpu")
+    for mode in ("zero", "duplicate"):
+        Wr = torch.zeros_like(host["W_r"]) if mode == "zero" else host["W_r"].clone()
+        if mode == "duplicate":
+            Wr[:, 40] = Wr[:, 3]
+        ctx = binding.context_for(w, route_path=binding.ROUTE_TENSOR)
+        idx = torch.empty((w.T, w.k), dtype=torch.int32, device="cuda")
+        gate = torch.empty((w.T, w.k), dtype=torch.float32, device="cuda")
+        binding.mop_moe_route(ctx, host["x"].cuda(), Wr.cuda(), None, idx, gate)
+        binding.mop_poll(ctx)
+        ref_idx, ref_gate = oracle.route(synth.bits(host["x"]), Wr.numpy(), None, w.k, w.score_fn, w.bias_mode)
+        assert np.array_equal(idx.cpu().numpy(), ref_idx), mode
+        assert np.all(np.abs(gate.cpu().numpy() - ref_gate) <= 1e-6 + 1e-5 * np.abs(ref_gate)), mode
+        if mode == "zero":
+            assert binding.mop_route_stats(ctx) == (w.T, w.T * w.E, 0)
+
+
+def test_tensor_core_scoring_refuses_shapes_it_cannot_take():
+    with pytest.raises(binding.MopError) as e:
+        binding.Context(64, 64, 40, 2, 64, route_path=binding.ROUTE_TENSOR)      # E not a multiple of 64
+    assert e.value.code == 6
