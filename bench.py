@@ -286,6 +286,8 @@ def bench_workload(w, args, steps, warmup, with_cpu_baseline):
     barrier = launch.barrier
 
     inp = synth.make_inputs(w, dev)
+    if args.chunks:
+        args.no_e2e = True      # the host-buffer entry points run the unchunked layer
     ctx = binding.context_for(w, device=local, host_io=0 if args.no_e2e else 2, gemm_path=args.gemm_path)
     buf = binding.LayerBuffers(w, device=dev)
     stream = torch.cuda.current_stream()
@@ -295,7 +297,21 @@ def bench_workload(w, args, steps, warmup, with_cpu_baseline):
         logits = torch.empty((w.T, w.E), dtype=torch.float32, device=dev)
         dW_r = torch.empty((w.d, w.E), dtype=torch.float32, device=dev)
 
+    chunk_ws = None
+    if args.chunks:
+        chunk_ws = torch.empty(binding.mop_moe_chunked_workspace_bytes(ctx, args.chunks, w.backward), dtype=torch.uint8,
+                               device=dev)
+
     def step():
+        if args.chunks:
+            binding.mop_moe_layer_fwd_chunked(ctx, args.chunks, inp["x"], inp["W_r"], inp["bias"], inp["W_gate"],
+                                              inp["W_up"], inp["W_down"], buf.idx, buf.gate, buf.counts, buf.offsets,
+                                              buf.perm_row, buf.row_src, buf.Y, chunk_ws, stream)
+            if w.backward:
+                binding.mop_moe_layer_bwd_chunked(ctx, args.chunks, inp["x"], inp["dY"], buf.gate, buf.offsets,
+                                                  buf.perm_row, buf.row_src, inp["W_gate"], inp["W_up"], inp["W_down"],
+                                                  buf.dX, buf.dW_gate, buf.dW_up, buf.dW_down, buf.dgate, chunk_ws, stream)
+            return
         if rbwd:   # the router keeps its logits for the backward
             binding.mop_moe_route(ctx, inp["x"], inp["W_r"], inp["bias"], buf.idx, buf.gate, logits, stream)
             binding.mop_moe_permute(ctx, inp["x"], buf.idx, buf.counts, buf.offsets, buf.perm_row, buf.row_src, buf.Xp,
@@ -446,6 +462,15 @@ def bench_workload(w, args, steps, warmup, with_cpu_baseline):
                "seconds": round(s1 + s2, 2),
                "sample": f"{1 + len(more)} median-load experts, {r1 + r2} rows: "
                          f"{'fwd+dgrad+wgrad' if w.backward else 'fwd'} of every row routed to them"}
+    # expert-contiguous activation buffers: whole layer (Xp, H, Yp; with a backward also the G, U stash and the
+    # context's dYp, dG, dU, gH, dXp) against one group of experts at a time plus the fp32 accumulator
+    M = w.T * w.k
+    full_bytes = M * (2 * w.d + w.f) * 2 + (M * (2 * w.f + 2 * w.d + 3 * w.f) * 2 if w.backward else 0)
+    memory = {"expert_contiguous_activation_bytes": full_bytes}
+    if args.chunks:
+        memory = {"chunks": args.chunks, "chunked_workspace_bytes": int(chunk_ws.numel()),
+                  "unchunked_expert_contiguous_activation_bytes": full_bytes,
+                  "ratio": chunk_ws.numel() / full_bytes}
     ctx.close()
     return {
         "metric": "moe_layer_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
@@ -457,7 +482,7 @@ def bench_workload(w, args, steps, warmup, with_cpu_baseline):
         "frac_of_bf16_peak_nominal": value / world / 2250.0,
         "frac_of_bf16_peak_measured": value / world / pk["bf16_tflops_sustained"],
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
-        "cpu_baseline": cpu,
+        "cpu_baseline": cpu, "memory": memory,
     }
 
 
@@ -478,12 +503,15 @@ def main():
                     help="also run the router backward (dgate -> dW_r, dX) in every step of a fwd+bwd workload")
     ap.add_argument("--gather", action="store_true",
                     help="forward-only workloads: up-projection gathers its rows from x (no permuted copy)")
+    ap.add_argument("--chunks", type=int, default=0,
+                    help="run the expert-chunked layer with this many groups of experts (buffers live for one group at a time)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra-workloads", action="store_true",
                     help="default invocation: skip the forward workloads that follow the headline")
     args = ap.parse_args()
-    extra = args.workload is None and args.shape is None and not args.no_extra_workloads and args.impl == "ours"
+    extra = (args.workload is None and args.shape is None and not args.no_extra_workloads and args.impl == "ours"
+             and not args.chunks)
     args.workload = args.workload or "c5_train"
     if args.workload in ("vocab_loss", "vocab_train"):
         return run_vocab(args)

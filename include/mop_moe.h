@@ -199,6 +199,33 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* ctx, const void* dY, const void* Xp, 
                                   const void* W_up, const void* W_down, void* dX, float* dW_gate, float* dW_up,
                                   float* dW_down, float* dgate, void* stream);
 
+/* Expert-chunked layer: the memory-lean form of Section 3.3, where only a fraction of the routed buffers is
+ * resident at any instant (the O(N k H + N_r I) activation term of Eq. 4 shrinks to one chunk of it).  The
+ * experts are cut into n_chunks groups of about T k / n_chunks rows each (a group ends at an expert boundary, so
+ * it holds at most one expert's rows more than its share); per group the rows are gathered from x, run through
+ * the expert feed-forward, and added to an fp32 accumulator of Y in group order (fixed order, no atomics:
+ * reproducible), which is rounded to bf16 once.  Xp, H and Yp therefore exist for one group at a time, in the
+ * caller's `workspace` of mop_moe_chunked_workspace_bytes(shape, n_chunks, with_backward) bytes (256-byte
+ * aligned).  The weights are read once, as in the unchunked layer.  The sum over a token's experts runs in
+ * expert order here and in score order in mop_moe_combine: Y agrees to fp32 summation order, not bit for bit.
+ * The backward keeps nothing of the forward: per group it gathers x and dY again, recomputes the up-projection,
+ * runs the data and weight gradients of the group (each expert's dW is written once), and accumulates dX the
+ * same way; experts without rows get zero gradients (or keep theirs when dw_accumulate is set).
+ * Needs the tensor-core path (MOP_ERR_UNSUPPORTED otherwise); 1 <= n_chunks <= 64.
+ * fwd: x, W_r, bias, W_* in; topk_idx, topk_gate, counts, offsets, perm_row, row_src, Y out (as in mop_moe_route,
+ * mop_moe_permute, mop_moe_combine).  bwd: x, dY, topk_gate, offsets, perm_row, row_src, W_* in; dX, dW_*, dgate out
+ * (as in mop_moe_expert_ffn_bwd); every intermediate lives in `workspace`, so any context of the shape will do. */
+size_t mop_moe_chunked_workspace_bytes(const mop_moe_shape* shape, int32_t n_chunks, int32_t with_backward);
+mop_status mop_moe_layer_fwd_chunked(mop_ctx* ctx, int32_t n_chunks, const void* x, const float* W_r, const float* bias,
+                                     const void* W_gate, const void* W_up, const void* W_down, int32_t* topk_idx,
+                                     float* topk_gate, int32_t* counts, int32_t* offsets, int32_t* perm_row,
+                                     int32_t* row_src, void* Y, void* workspace, void* stream);
+mop_status mop_moe_layer_bwd_chunked(mop_ctx* ctx, int32_t n_chunks, const void* x, const void* dY,
+                                     const float* topk_gate, const int32_t* offsets, const int32_t* perm_row,
+                                     const int32_t* row_src, const void* W_gate, const void* W_up, const void* W_down,
+                                     void* dX, float* dW_gate, float* dW_up, float* dW_down, float* dgate,
+                                     void* workspace, void* stream);
+
 /* Router backward with the selection held fixed (Section 2.1's router, differentiated through the
  * gate renormalisation and the score function; the step on either side of the expert path).
  *   softmax:  dz_j = g_j (dgate_j - sum_l g_l dgate_l)

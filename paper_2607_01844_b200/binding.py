@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.mop_moe_train_step_host_async.argtypes = [_P] * 15
         L.mop_host_drain.argtypes = [_P] * 2
         L.mop_moe_route_bwd.argtypes = [_P] * 14
+        L.mop_moe_chunked_workspace_bytes.argtypes = [ctypes.POINTER(MopShape), ctypes.c_int32, ctypes.c_int32]
+        L.mop_moe_chunked_workspace_bytes.restype = ctypes.c_size_t
+        L.mop_moe_layer_fwd_chunked.argtypes = [_P, ctypes.c_int32] + [_P] * 15
+        L.mop_moe_layer_bwd_chunked.argtypes = [_P, ctypes.c_int32] + [_P] * 16
         L.mop_moe_train_step_host.argtypes = [_P] * 15
         L.mop_moe_permute_static.argtypes = [ctypes.c_int] + [ctypes.c_int32] * 4 + [_P] * 8
         L.mop_vocab_workspace_bytes.argtypes = [ctypes.c_int32] * 3
@@ -213,6 +217,29 @@ def mop_moe_route_bwd(ctx, logits, bias, topk_idx, topk_gate, dgate, Xp, offsets
            lib().mop_moe_route_bwd(ctx.handle, _ptr(logits), _ptr(bias), _ptr(topk_idx), _ptr(topk_gate), _ptr(dgate),
                                    _ptr(Xp), _ptr(offsets), _ptr(perm_row), _ptr(W_r), _ptr(dW_r), _ptr(dbias),
                                    _ptr(dX), _stream(stream)))
+
+
+def mop_moe_chunked_workspace_bytes(ctx, n_chunks, with_backward=False):
+    return lib().mop_moe_chunked_workspace_bytes(ctypes.byref(ctx.shape), n_chunks, int(with_backward))
+
+
+def mop_moe_layer_fwd_chunked(ctx, n_chunks, x, W_r, bias, W_gate, W_up, W_down, topk_idx, topk_gate, counts, offsets,
+                              perm_row, row_src, Y, workspace, stream=None):
+    """Whole forward with the expert-contiguous buffers live for one group of experts at a time."""
+    _check("mop_moe_layer_fwd_chunked",
+           lib().mop_moe_layer_fwd_chunked(ctx.handle, n_chunks, _ptr(x), _ptr(W_r), _ptr(bias), _ptr(W_gate), _ptr(W_up),
+                                           _ptr(W_down), _ptr(topk_idx), _ptr(topk_gate), _ptr(counts), _ptr(offsets),
+                                           _ptr(perm_row), _ptr(row_src), _ptr(Y), _ptr(workspace), _stream(stream)))
+
+
+def mop_moe_layer_bwd_chunked(ctx, n_chunks, x, dY, topk_gate, offsets, perm_row, row_src, W_gate, W_up, W_down, dX,
+                              dW_gate, dW_up, dW_down, dgate, workspace, stream=None):
+    """Whole backward of the chunked layer (recomputes the up-projection per group of experts)."""
+    _check("mop_moe_layer_bwd_chunked",
+           lib().mop_moe_layer_bwd_chunked(ctx.handle, n_chunks, _ptr(x), _ptr(dY), _ptr(topk_gate), _ptr(offsets),
+                                           _ptr(perm_row), _ptr(row_src), _ptr(W_gate), _ptr(W_up), _ptr(W_down),
+                                           _ptr(dX), _ptr(dW_gate), _ptr(dW_up), _ptr(dW_down), _ptr(dgate),
+                                           _ptr(workspace), _stream(stream)))
 
 
 def mop_moe_forward_host(ctx, x_host, W_r, bias, W_gate, W_up, W_down, Y_host, idx_host=None, gate_host=None,

@@ -58,7 +58,7 @@ inline mop_status tc_up_only(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int3
 inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
                                   int* launches, bool with_down) {
     const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
+    const uint64_t M = tc_rows(p);
     mop_status r;
     // Tokens-on-N kernels: fwd_tn bit 0 = up-projection, bit 1 = down-projection (see tc_plan_policy)
     const bool gather = a.x_gather != nullptr;
@@ -109,11 +109,11 @@ inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles,
 inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st,
                              int* launches, int* ntile_part) {
     const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
+    const uint64_t M = tc_rows(p);
     *ntile_part = ceil_div(s.f, 256);
     if (M == 0) {
         // no rows at all: gradients are zero unless accumulating
-        if (!a.accumulate) {
+        if (!a.accumulate && !a.keep_empty) {
             const size_t n = (size_t)s.E * s.d * s.f * 4;
             if (cudaMemsetAsync(a.dW_gate, 0, n, st) != cudaSuccess || cudaMemsetAsync(a.dW_up, 0, n, st) != cudaSuccess ||
                 cudaMemsetAsync(a.dW_down, 0, n, st) != cudaSuccess)
@@ -171,14 +171,14 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
     {   // WD: dW_down[e] = (gate H)_e^T dYp_e
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = ceil_div(s.d, 256); g.tiles_m_fixed = ceil_div(s.f, TC_BM); g.Mfix = s.f; g.N = s.d;
-        g.ep.outf = a.dW_down; g.ep.accumulate = a.accumulate;
+        g.ep.outf = a.dW_down; g.ep.accumulate = a.accumulate; g.keep_empty = a.keep_empty;
         if ((r = tc_launch<TC_WD>(p, "gemm_wgrad_down", mgH, mgH, mdYpB, mdYpB, moWd, moWd, g, st)) != MOP_OK) return r;
         ++*launches;
     }
     {   // WGU: dW_gate[e] = Xp_e^T dG_e and dW_up[e] = Xp_e^T dU_e: per m-block the n-tiles of dW_gate, then those of dW_up
         TcArgs g = tc_base_args(p, a.offsets, tiles, status);
         g.tiles_n = 2 * ceil_div(s.f, 256); g.tiles_m_fixed = ceil_div(s.d, TC_BM); g.Mfix = s.d; g.N = s.f;
-        g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate;
+        g.ep.outf = a.dW_gate; g.outf1 = a.dW_up; g.ep.accumulate = a.accumulate; g.keep_empty = a.keep_empty;
         if ((r = tc_launch<TC_WGU>(p, "gemm_wgrad_gate_up", mXpA, mXpA, mdGB, mdUB, moWg, moWu, g, st)) != MOP_OK) return r;
         ++*launches;
     }

@@ -84,6 +84,7 @@ struct TcArgs {
     int32_t* status;
     EpiArgs ep;
     float* outf1;            // WGU: second output tensor
+    int keep_empty;          // weight gradients: leave the gradients of experts without rows untouched
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -714,7 +715,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
             if constexpr (Tr::RAGGED_K) {
                 if (ti.skip) {
                     // expert without rows: its gradient is zero (or unchanged when accumulating)
-                    if (!args.ep.accumulate && half == 0 && ti.m0 + r < args.Mfix) {
+                    if (!args.ep.accumulate && !args.keep_empty && half == 0 && ti.m0 + r < args.Mfix) {
                         const size_t ro = ((size_t)ti.e * args.Mfix + ti.m0 + r) * args.N;
                         float* dst = (Tr::SEL_B && ti.sel) ? args.outf1 : args.ep.outf;
                         for (int c = 0; c < TC_BN; c += 4)
@@ -880,6 +881,7 @@ struct TcPlan {
     mop_moe_shape s;
     void* encode;   // cuTensorMapEncodeTiled
     int pairs;      // schedule of the token-row kinds (see gemm_host.cuh)
+    long long rows_override;   // > 0: the row buffers of this call hold this many rows (an expert chunk), not T*k
     int fwd_tn;     // GEMMs on the tokens-on-N kernels: bit 0 up-projection, bit 1 down-projection, bit 2 dgrad of the up-projection, bit 3 dgrad of the down-projection
     Profiler* prof;
 };
@@ -896,9 +898,13 @@ struct TcBwdArgs {
     const bf16 *W_gate, *W_up, *W_down;
     bf16 *dG, *dU, *gH, *dXp; float* part;
     float *dW_gate, *dW_up, *dW_down; int accumulate;
+    int keep_empty;   // experts without rows (in this call's offsets) keep their gradients: expert-chunked backward
 };
 
 inline bool tc_shape_supported(int d, int f) { return d % 64 == 0 && f % 64 == 0; }
+inline uint64_t tc_rows(const TcPlan* p) {
+    return p->rows_override > 0 ? (uint64_t)p->rows_override : (uint64_t)p->s.T * p->s.k;
+}
 inline size_t tc_tile_table_bytes(int M, int E) { return ((size_t)M / TC_BM + E + 8) * sizeof(int4) + 256; }
 
 typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -916,6 +922,7 @@ inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count, 
     p->sm_count = sm_count;
     p->prof = prof;
     p->s = s;
+    p->rows_override = 0;
     cudaDriverEntryPointQueryResult q;
     void* fn = nullptr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||

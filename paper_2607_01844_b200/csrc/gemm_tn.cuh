@@ -508,7 +508,7 @@ inline TnArgs tn_base_args(int32_t* tiles, int32_t* status) {
 // Up-projection + SwiGLU on the tokens-on-N kernel (`tiles` holds the token-tile table).
 inline mop_status tn_up_swiglu(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
     const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
+    const uint64_t M = tc_rows(p);
     CUtensorMap mXp, mWg, mWu;
     if (!tc_map_2d(p, &mXp, a.Xp, M, s.d, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 1, 128) ||
         !tc_map_chunked_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 1, 128))
@@ -543,7 +543,7 @@ inline mop_status tn_up_swiglu_gather(TcPlan* p, const bf16* x, const TcFwdArgs&
 // Down-projection + gate on the tokens-on-N kernel.
 inline mop_status tn_down_gate(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
     const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
+    const uint64_t M = tc_rows(p);
     CUtensorMap mH, mWd;
     if (!tc_map_2d(p, &mH, a.H, M, s.f, TN_BOX_ROWS) || !tc_map_chunked_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 2, 128))
         return MOP_ERR_CUDA;
@@ -559,7 +559,7 @@ inline mop_status tn_down_gate(TcPlan* p, const TcFwdArgs& a, int32_t* tiles, in
 // Data gradient of the up-projection on the tokens-on-N kernel: dXp = dG W_gate^T + dU W_up^T.
 inline mop_status tn_dgrad_gate_up(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
     const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
+    const uint64_t M = tc_rows(p);
     CUtensorMap mWg, mWu, mdG, mdU;
     if (!tc_map_3d(p, &mWg, a.W_gate, s.E, s.d, s.f, 128) || !tc_map_3d(p, &mWu, a.W_up, s.E, s.d, s.f, 128) ||
         !tc_map_2d(p, &mdG, a.dG, M, s.f, TN_BOX_ROWS) || !tc_map_2d(p, &mdU, a.dU, M, s.f, TN_BOX_ROWS))
@@ -577,7 +577,7 @@ inline mop_status tn_dgrad_gate_up(TcPlan* p, const TcBwdArgs& a, int32_t* tiles
 // Writes one dgate partial per 32 columns of f (part[f / 32][row]).
 inline mop_status tn_dgrad_down(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int32_t* status, cudaStream_t st) {
     const mop_moe_shape& s = p->s;
-    const uint64_t M = (uint64_t)s.T * s.k;
+    const uint64_t M = tc_rows(p);
     CUtensorMap mWd, mdYp;
     if (!tc_map_3d(p, &mWd, a.W_down, s.E, s.f, s.d, 128) || !tc_map_2d(p, &mdYp, a.dYp, M, s.d, TN_BOX_ROWS))
         return MOP_ERR_CUDA;

@@ -830,6 +830,206 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
     return mop_moe_combine(c, c->dXp, perm_row, dX, stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Expert-chunked layer: the expert-contiguous buffers (Xp, H, Yp and the backward's intermediates) exist
+// for one chunk of experts at a time, in a workspace the caller provides.
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct ChunkLayout {
+    size_t off_c, row_src_c, perm_c, bounds, Xp, H, Yp, acc, G, U, dYp, dG, dU, gH, dXp, part, total;
+    long long cap;   // rows of a chunk's buffers
+};
+ChunkLayout chunk_layout(const mop_moe_shape& s, int C, int bwd) {
+    ChunkLayout L{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o += align_up(bytes); return r; };
+    const size_t T = s.T, d = s.d, E = s.E, k = s.k, f = s.f, M = T * k;
+    // a chunk ends at an expert boundary at or past its share of the rows: at most one expert more than M / C
+    size_t cap = (M + C - 1) / C + T;
+    if (cap > M) cap = M;
+    cap = (cap + 15) / 16 * 16;
+    L.cap = (long long)cap;
+    L.off_c = take((E + 1) * 4);
+    L.row_src_c = take(cap * 4 + 16);
+    L.perm_c = take(M * 4 + 16);
+    L.bounds = take(16);
+    L.Xp = take(cap * d * 2);
+    L.H = take(cap * f * 2);
+    L.Yp = take(cap * d * 2);
+    L.acc = take(T * d * 4);
+    if (bwd) {
+        L.G = take(cap * f * 2);
+        L.U = take(cap * f * 2);
+        L.dYp = take(cap * d * 2);
+        L.dG = take(cap * f * 2);
+        L.dU = take(cap * f * 2);
+        L.gH = take(cap * f * 2);
+        L.dXp = take(cap * d * 2);
+        L.part = take((size_t)part_tiles(s) * cap * 4);
+    }
+    L.total = o;
+    return L;
+}
+mop_status chunk_check(mop_ctx* c, int32_t n_chunks, const void* workspace) {
+    if (!c) return MOP_ERR_INVALID_ARG;
+    if (n_chunks < 1 || n_chunks > 64) return MOP_ERR_INVALID_ARG;
+    if (!workspace) return MOP_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MOP_ERR_ALIGN;
+    if (!use_tensor(c)) return MOP_ERR_UNSUPPORTED;    // the chunked layer runs on the tensor-core kernels only
+    return MOP_OK;
+}
+// tables, gathered inputs of chunk i
+mop_status chunk_begin(mop_ctx* c, const ChunkLayout& L, char* w, int i, int C, const void* src, size_t dst_off,
+                       const int32_t* offsets, const int32_t* perm_row, const int32_t* row_src, bool tables,
+                       cudaStream_t st) {
+    const mop_moe_shape& s = c->s;
+    const int M = s.T * s.k;
+    int32_t* off_c = reinterpret_cast<int32_t*>(w + L.off_c);
+    int32_t* row_src_c = reinterpret_cast<int32_t*>(w + L.row_src_c);
+    int32_t* perm_c = reinterpret_cast<int32_t*>(w + L.perm_c);
+    int32_t* bounds = reinterpret_cast<int32_t*>(w + L.bounds);
+    mop_status r;
+    if (tables) {
+        LAUNCH(c, "chunk_tables", st,
+               chunk_tables_kernel<<<min(ceil_div(M, 256), c->sm_count * 4), 256, 0, st>>>(
+                   offsets, row_src, perm_row, off_c, row_src_c, perm_c, bounds, s.E, M, i, C));
+        if ((r = after_launch(c)) != MOP_OK) return r;
+    }
+    LAUNCH(c, "chunk_gather_rows", st,
+           gather_rows_kernel<<<c->sm_count * 8, 256, 0, st>>>(static_cast<const uint4*>(src),
+                                                               reinterpret_cast<uint4*>(w + dst_off), row_src_c, bounds,
+                                                               s.k, s.d / 8));
+    return after_launch(c);
+}
+}  // namespace
+
+size_t mop_moe_chunked_workspace_bytes(const mop_moe_shape* shape, int32_t n_chunks, int32_t with_backward) {
+    if (check_shape(shape) != MOP_OK || n_chunks < 1 || n_chunks > 64) return 0;
+    return chunk_layout(*shape, n_chunks, with_backward).total;
+}
+
+mop_status mop_moe_layer_fwd_chunked(mop_ctx* c, int32_t n_chunks, const void* x, const float* W_r, const float* bias,
+                                     const void* W_gate, const void* W_up, const void* W_down, int32_t* topk_idx,
+                                     float* topk_gate, int32_t* counts, int32_t* offsets, int32_t* perm_row,
+                                     int32_t* row_src, void* Y, void* workspace, void* stream) {
+    mop_status r = chunk_check(c, n_chunks, workspace);
+    if (r != MOP_OK) return r;
+    REQ_PTR_T(x); REQ_PTR(W_r); REQ_PTR(W_gate); REQ_PTR(W_up); REQ_PTR(W_down); REQ_PTR_T(topk_idx); REQ_PTR_T(topk_gate);
+    REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR_T(perm_row); REQ_PTR_T(row_src); REQ_PTR_T(Y);
+    const mop_moe_shape& s = c->s;
+    if ((r = mop_moe_route(c, x, W_r, bias, topk_idx, topk_gate, nullptr, stream)) != MOP_OK) return r;
+    if ((r = mop_moe_permute(c, nullptr, topk_idx, counts, offsets, perm_row, row_src, nullptr, stream)) != MOP_OK) return r;
+    if (s.T == 0) return MOP_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const ChunkLayout L = chunk_layout(s, n_chunks, 0);
+    char* w = static_cast<char*>(workspace);
+    const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
+    c->plan.rows_override = L.cap;
+    for (int i = 0; i < n_chunks && r == MOP_OK; ++i) {
+        if ((r = chunk_begin(c, L, w, i, n_chunks, x, L.Xp, offsets, perm_row, row_src, true, st)) != MOP_OK) break;
+        TcFwdArgs a{};
+        a.Xp = reinterpret_cast<const bf16*>(w + L.Xp); a.offsets = reinterpret_cast<const int32_t*>(w + L.off_c);
+        a.row_src = reinterpret_cast<const int32_t*>(w + L.row_src_c); a.gate = topk_gate;
+        a.W_gate = static_cast<const bf16*>(W_gate); a.W_up = static_cast<const bf16*>(W_up);
+        a.W_down = static_cast<const bf16*>(W_down);
+        a.H = reinterpret_cast<bf16*>(w + L.H); a.Yp = reinterpret_cast<bf16*>(w + L.Yp);
+        int n = 0;
+        r = tc_ffn_fwd(&c->plan, a, c->tiles, c->status, st, &n);
+        c->launches += n;
+        if (r != MOP_OK) break;
+        LAUNCH(c, "chunk_combine_acc", st,
+               combine_acc_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(w + L.Yp),
+                                                         reinterpret_cast<const int32_t*>(w + L.perm_c),
+                                                         reinterpret_cast<float4*>(w + L.acc), static_cast<uint4*>(Y), s.T,
+                                                         s.k, s.d / 8, i == 0, i == n_chunks - 1));
+        r = after_launch(c);
+    }
+    c->plan.rows_override = 0;
+    return r;
+}
+
+mop_status mop_moe_layer_bwd_chunked(mop_ctx* c, int32_t n_chunks, const void* x, const void* dY,
+                                     const float* topk_gate, const int32_t* offsets, const int32_t* perm_row,
+                                     const int32_t* row_src, const void* W_gate, const void* W_up, const void* W_down,
+                                     void* dX, float* dW_gate, float* dW_up, float* dW_down, float* dgate,
+                                     void* workspace, void* stream) {
+    mop_status r = chunk_check(c, n_chunks, workspace);
+    if (r != MOP_OK) return r;
+    REQ_PTR_T(x); REQ_PTR_T(dY); REQ_PTR_T(topk_gate); REQ_PTR(offsets); REQ_PTR_T(perm_row); REQ_PTR_T(row_src);
+    REQ_PTR(W_gate); REQ_PTR(W_up); REQ_PTR(W_down); REQ_PTR_T(dX); REQ_PTR(dW_gate); REQ_PTR(dW_up); REQ_PTR(dW_down);
+    REQ_PTR_T(dgate);
+    const mop_moe_shape& s = c->s;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return MOP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t wvec = (size_t)s.d * s.f / 4;
+    if (s.T == 0) {
+        if (!s.dw_accumulate) {
+            const size_t n = (size_t)s.E * s.d * s.f * 4;
+            CUDA_OK(cudaMemsetAsync(dW_gate, 0, n, st)); CUDA_OK(cudaMemsetAsync(dW_up, 0, n, st));
+            CUDA_OK(cudaMemsetAsync(dW_down, 0, n, st));
+        }
+        return MOP_OK;
+    }
+    const ChunkLayout L = chunk_layout(s, n_chunks, 1);
+    char* w = static_cast<char*>(workspace);
+    const int M = s.T * s.k;
+    const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
+    c->plan.rows_override = L.cap;
+    for (int i = 0; i < n_chunks && r == MOP_OK; ++i) {
+        // the chunk's inputs again, and its up-projection recomputed (nothing of the forward was kept)
+        if ((r = chunk_begin(c, L, w, i, n_chunks, x, L.Xp, offsets, perm_row, row_src, true, st)) != MOP_OK) break;
+        if ((r = chunk_begin(c, L, w, i, n_chunks, dY, L.dYp, offsets, perm_row, row_src, false, st)) != MOP_OK) break;
+        const int32_t* off_c = reinterpret_cast<const int32_t*>(w + L.off_c);
+        const int32_t* row_src_c = reinterpret_cast<const int32_t*>(w + L.row_src_c);
+        TcFwdArgs fa{};
+        fa.Xp = reinterpret_cast<const bf16*>(w + L.Xp); fa.offsets = off_c;
+        fa.W_gate = static_cast<const bf16*>(W_gate); fa.W_up = static_cast<const bf16*>(W_up);
+        fa.G_save = reinterpret_cast<bf16*>(w + L.G); fa.U_save = reinterpret_cast<bf16*>(w + L.U);
+        fa.H = reinterpret_cast<bf16*>(w + L.H);
+        int n = 0;
+        r = tc_up_only(&c->plan, fa, c->tiles, c->status, st, &n);
+        c->launches += n;
+        if (r != MOP_OK) break;
+        TcBwdArgs a{};
+        a.dYp = reinterpret_cast<const bf16*>(w + L.dYp); a.Xp = fa.Xp; a.G_save = fa.G_save; a.U_save = fa.U_save; a.H = fa.H;
+        a.offsets = off_c; a.row_src = row_src_c; a.gate = topk_gate;
+        a.W_gate = fa.W_gate; a.W_up = fa.W_up; a.W_down = static_cast<const bf16*>(W_down);
+        a.dG = reinterpret_cast<bf16*>(w + L.dG); a.dU = reinterpret_cast<bf16*>(w + L.dU);
+        a.gH = reinterpret_cast<bf16*>(w + L.gH); a.dXp = reinterpret_cast<bf16*>(w + L.dXp);
+        a.part = reinterpret_cast<float*>(w + L.part);
+        a.dW_gate = dW_gate; a.dW_up = dW_up; a.dW_down = dW_down; a.accumulate = s.dw_accumulate; a.keep_empty = 1;
+        int ntile_part = 0;
+        n = 0;
+        r = tc_ffn_bwd(&c->plan, a, c->tiles, c->status, st, &n, &ntile_part);
+        c->launches += n;
+        if (r != MOP_OK) break;
+        LAUNCH(c, "chunk_dgate_reduce", st,
+               dgate_reduce_chunk_kernel<<<ceil_div(M, 256), 256, 0, st>>>(a.part, reinterpret_cast<const int32_t*>(w + L.perm_c),
+                                                                           dgate, M, (int)L.cap, ntile_part));
+        if ((r = after_launch(c)) != MOP_OK) break;
+        LAUNCH(c, "chunk_combine_acc", st,
+               combine_acc_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(w + L.dXp),
+                                                         reinterpret_cast<const int32_t*>(w + L.perm_c),
+                                                         reinterpret_cast<float4*>(w + L.acc), static_cast<uint4*>(dX), s.T,
+                                                         s.k, s.d / 8, i == 0, i == n_chunks - 1));
+        r = after_launch(c);
+    }
+    c->plan.rows_override = 0;
+    if (r != MOP_OK) return r;
+    if (!s.dw_accumulate) {   // experts that received no row: zero gradients
+        dim3 gz((unsigned)min((size_t)64, (wvec + 255) / 256), s.E);
+        LAUNCH(c, "chunk_zero_empty_experts", st,
+               zero_empty_experts_kernel<<<gz, 256, 0, st>>>(offsets, reinterpret_cast<float4*>(dW_gate),
+                                                             reinterpret_cast<float4*>(dW_up),
+                                                             reinterpret_cast<float4*>(dW_down), wvec));
+        r = after_launch(c);
+    }
+    return r;
+}
+
 mop_status mop_moe_route_bwd(mop_ctx* c, const float* logits, const float* bias, const int32_t* topk_idx,
                              const float* topk_gate, const float* dgate, const void* Xp, const int32_t* offsets,
                              const int32_t* perm_row, const float* W_r, float* dW_r, float* dbias_opt, void* dX,

@@ -196,4 +196,125 @@ __global__ void dgate_reduce_kernel(const float* __restrict__ part, const int32_
     dgate[a] = s;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Expert-chunked layer (only a fraction of the expert-contiguous buffers is live at a time).
+// Chunk i of C takes the experts [eb(i), eb(i+1)) where eb(i) is the first expert whose first row is
+// at or past ceil(i M / C): C chunks of at most ceil(M / C) + (rows of one expert) rows each.
+// ---------------------------------------------------------------------------------------------
+
+// Tables of one chunk: off_c[e] = first row of expert e inside the chunk's buffers (experts outside the
+// chunk get no rows), row_src_c[r] = assignment of chunk row r, perm_c[a] = chunk row of assignment a or -1.
+// bounds[0] = first row of the chunk in the whole layer, bounds[1] = its rows.
+__global__ void __launch_bounds__(256) chunk_tables_kernel(const int32_t* __restrict__ offsets,
+                                                           const int32_t* __restrict__ row_src,
+                                                           const int32_t* __restrict__ perm_row,
+                                                           int32_t* __restrict__ off_c, int32_t* __restrict__ row_src_c,
+                                                           int32_t* __restrict__ perm_c, int32_t* __restrict__ bounds,
+                                                           int E, int M, int chunk, int n_chunks) {
+    __shared__ int32_t s_lo, s_hi;
+    if (threadIdx.x == 0) {
+        const long long t0 = ((long long)chunk * M + n_chunks - 1) / n_chunks;
+        const long long t1 = ((long long)(chunk + 1) * M + n_chunks - 1) / n_chunks;
+        int e0 = 0, e1 = 0;
+        while (e0 < E && offsets[e0] < t0) ++e0;          // E <= 1024: a short serial search
+        e1 = e0;
+        if (chunk + 1 == n_chunks) e1 = E;
+        else while (e1 < E && offsets[e1] < t1) ++e1;
+        s_lo = offsets[e0];
+        s_hi = offsets[e1];
+    }
+    __syncthreads();
+    const int lo = s_lo, hi = s_hi;
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsz = gridDim.x * blockDim.x;
+    if (gtid == 0) { bounds[0] = lo; bounds[1] = hi - lo; }
+    for (int e = gtid; e <= E; e += gsz) off_c[e] = min(max(offsets[e], lo), hi) - lo;
+    for (int r = gtid; r < hi - lo; r += gsz) row_src_c[r] = row_src[lo + r];
+    for (int a = gtid; a < M; a += gsz) {
+        const int32_t p = perm_row[a];
+        perm_c[a] = (p >= lo && p < hi) ? p - lo : -1;
+    }
+}
+
+// Xp_c[r,:] = x[row_src_c[r] / k, :] for the rows of a chunk (one warp per row, 16-byte vectors).
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
+                                                          const int32_t* __restrict__ row_src_c,
+                                                          const int32_t* __restrict__ bounds, int k, int vec_per_row) {
+    const int rows = bounds[1];
+    const int lane = threadIdx.x % 32, wpb = blockDim.x / 32;
+    for (int r = blockIdx.x * wpb + threadIdx.x / 32; r < rows; r += gridDim.x * wpb) {
+        const uint4* s = src + (size_t)(row_src_c[r] / k) * vec_per_row;
+        uint4* o = dst + (size_t)r * vec_per_row;
+        for (int c = lane; c < vec_per_row; c += 32) __stcs(o + c, __ldg(s + c));
+    }
+}
+
+// Accumulating combine: acc[t,:] (+)= sum_j Yp_c[perm_c[t*k+j], :] over the token's rows inside the chunk
+// (fp32, j ascending; chunks are added in chunk order, so the result is reproducible).  first: acc is
+// written, not read; last: the sum is rounded once to bf16 into out instead of going back to acc.
+__global__ void __launch_bounds__(256) combine_acc_kernel(const uint4* __restrict__ Yp_c,
+                                                          const int32_t* __restrict__ perm_c, float4* __restrict__ acc,
+                                                          uint4* __restrict__ out, int T, int k, int vec_per_row,
+                                                          int first, int last) {
+    const int wpb = blockDim.x / 32, lane = threadIdx.x % 32;
+    for (int t = blockIdx.x * wpb + threadIdx.x / 32; t < T; t += gridDim.x * wpb) {
+        int32_t myrow = -1;
+        if (lane < k) myrow = perm_c[(size_t)t * k + lane];
+        const bool any = __any_sync(0xffffffffu, myrow >= 0);
+        if (!any && !first && !last) continue;              // nothing of this token in the chunk
+        for (int c = lane; c < vec_per_row; c += 32) {
+            float a[8];
+            float4* ap = acc + ((size_t)t * vec_per_row + c) * 2;
+            if (first) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a[i] = 0.0f;
+            } else {
+                const float4 a0 = ap[0], a1 = ap[1];
+                a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+            }
+            for (int j = 0; j < k; ++j) {
+                const int32_t p = __shfl_sync(0xffffffffu, myrow, j);
+                if (p < 0) continue;
+                const uint4 v = __ldcs(Yp_c + (size_t)p * vec_per_row + c);
+                a[0] += bf16_lo(v.x); a[1] += bf16_hi(v.x); a[2] += bf16_lo(v.y); a[3] += bf16_hi(v.y);
+                a[4] += bf16_lo(v.z); a[5] += bf16_hi(v.z); a[6] += bf16_lo(v.w); a[7] += bf16_hi(v.w);
+            }
+            if (last) {
+                uint4 o;
+                o.x = pack_bf16x2(a[0], a[1]); o.y = pack_bf16x2(a[2], a[3]);
+                o.z = pack_bf16x2(a[4], a[5]); o.w = pack_bf16x2(a[6], a[7]);
+                out[(size_t)t * vec_per_row + c] = o;
+            } else {
+                ap[0] = make_float4(a[0], a[1], a[2], a[3]);
+                ap[1] = make_float4(a[4], a[5], a[6], a[7]);
+            }
+        }
+    }
+}
+
+// dgate of the assignments that lie inside the chunk (others are left alone).
+__global__ void dgate_reduce_chunk_kernel(const float* __restrict__ part, const int32_t* __restrict__ perm_c,
+                                          float* __restrict__ dgate, int M, int rows_pitch, int ntiles) {
+    const int a = blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= M) return;
+    const int32_t p = perm_c[a];
+    if (p < 0) return;
+    float s = 0.0f;
+    for (int n = 0; n < ntiles; ++n) s += part[(size_t)n * rows_pitch + p];
+    dgate[a] = s;
+}
+
+// Zero the weight gradients of the experts that received no row (the chunked backward writes only experts with rows).
+__global__ void __launch_bounds__(256) zero_empty_experts_kernel(const int32_t* __restrict__ offsets,
+                                                                float4* __restrict__ dWg, float4* __restrict__ dWu,
+                                                                float4* __restrict__ dWd, size_t vec_per_expert) {
+    const int e = blockIdx.y;
+    if (offsets[e + 1] > offsets[e]) return;
+    const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < vec_per_expert; i += (size_t)gridDim.x * blockDim.x) {
+        dWg[e * vec_per_expert + i] = z;
+        dWu[e * vec_per_expert + i] = z;
+        dWd[e * vec_per_expert + i] = z;
+    }
+}
+
 }  // namespace mop
