@@ -74,7 +74,7 @@ def kernel_work(w, counts):
         "route_select": (0, T * E * 4 + T * k * 8),
         # tensor-core scoring: three bf16 pieces of W_r, x read once, logits written and read back once
         "route_score_tc": (3 * 2 * T * d * E, T * d * 2 + 3 * d * E * 2 + T * E * 4),
-        "route_select_fast": (0, T * E * 4 + T * k * 8),
+        "route_select_screen": (0, T * E * 4 + T * k * 8),
         "route_bwd_dwr": (2 * M * d, M * d * 2 + M * 4 + d * E * 4),
         "route_bwd_dx": (2 * M * d, 2 * T * d * 2 + T * k * 8 + d * E * 4),
         "permute_scatter_rows": (0, T * d * 2 + M * d * 2 + M * 4),

@@ -11,8 +11,6 @@
 //   VL   Y = X W_voc (never stored)               online log-sum-exp partials         dense M
 //   VP   dY = g ([v = t] - exp(X W_voc - lse))     bf16, one block of vocabulary columns dense M
 //   VX   dX += dY W_voc^T over that block          fp32 read-modify-write              dense M
-//   RS   z~ = x (W_hi + W_mid + W_lo)              router logits from three bf16 pieces of W_r (three K
-//                                                  phases into one accumulator), fp32 store   dense M
 // CTA tile 128 x 256 (one tcgen05.mma.cta_group::1 of M=128, N=256, K=16 per 32 bytes of K),
 // K step 64 per pipeline stage, 4 stages, two 256-column accumulators in TMEM so that the
 // epilogue of tile i overlaps the main loop of tile i+1.
@@ -28,7 +26,7 @@
 
 namespace mop {
 
-enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5, TC_VL = 6, TC_VP = 7, TC_VX = 8, TC_RS = 9 };
+enum : int { TC_F1 = 0, TC_F2 = 1, TC_B2 = 2, TC_B4 = 3, TC_WD = 4, TC_WGU = 5, TC_VL = 6, TC_VP = 7, TC_VX = 8 };
 
 constexpr int TC_BM = 128, TC_BN = 256, TC_BK = 64;
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // 16 KiB
@@ -49,17 +47,12 @@ struct TcTraits {
     static constexpr bool SEL_B = (KIND == TC_WGU);
     static constexpr bool RAGGED_K = A_MN;
     static constexpr bool B_WEIGHT = !RAGGED_K;                       // B is an [E, ., .] weight tensor
-    static constexpr int PHASES = (KIND == TC_B4) ? 2 : (KIND == TC_RS) ? 3 : 1;
+    static constexpr int PHASES = (KIND == TC_B4) ? 2 : 1;
     static constexpr int N_PER_TILE = DUAL_B ? 128 : 256;             // output columns per tensor per tile
     // Weight gradients have a short K loop (the expert's rows) and a 128 KiB fp32 tile to write, so
     // they run eight epilogue warps (two per TMEM lane quarter, 128 columns each).
     static constexpr int STAGES = RAGGED_K ? 3 : 4;
-    static constexpr int EPI_WARPS = (RAGGED_K || KIND == TC_RS) ? 8 : 4;
-    // RS sums its K loop in segments: the tensor core accumulates SEG_KB blocks of 64 into a fresh accumulator,
-    // the epilogue adds the segment to fp32 registers (round to nearest).  The tensor core's own accumulation
-    // truncates, which over the 1344 updates of d = 7168 x 3 pieces would bias the logits by 2e-4; over 32
-    // updates per segment the bias stays below the rounding noise of the reference chain itself.
-    static constexpr int SEG_KB = (KIND == TC_RS) ? 8 : 0;
+    static constexpr int EPI_WARPS = RAGGED_K ? 8 : 4;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
     static constexpr int STORE_BYTES = RAGGED_K ? 4 * 16384 : 0;   // two 128-row x 32-column fp32 store boxes per half
     static constexpr int SMEM_BYTES = STAGES * TC_STAGE_BYTES + 1024 /*align*/ + TC_BAR_BYTES + STORE_BYTES;
@@ -576,8 +569,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                         // chunked maps {64, rows, cols/64 [, E]}: the 64-wide column chunks of the tile arrive
                         // chunk-major in one copy per tensor (four chunks, or two each of two tensors)
                         if constexpr (Tr::B_WEIGHT) {
-                            // RS: the "expert" coordinate of the weight map selects the piece of W_r
-                            tma_load_4d(sB, &tmB0, fb, 0, k0, n0 >> 6, KIND == TC_RS ? ph : ti.e);
+                            tma_load_4d(sB, &tmB0, fb, 0, k0, n0 >> 6, ti.e);
                             if constexpr (Tr::DUAL_B) tma_load_4d(sB + 2 * TC_CHUNK_BYTES, &tmB1, fb, 0, k0, n0 >> 6, ti.e);
                         } else {
                             const int krow = ti.row0 + kb * TC_BK;
@@ -610,7 +602,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                     const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
                     if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag, args.status, STATUS_WAIT_TMEM_EMPTY)) break;
                     tc_fence_after();
-                    uint32_t d_tmem = tmem_base + (uint32_t)buf * TC_BN;
+                    const uint32_t d_tmem = tmem_base + (uint32_t)buf * TC_BN;
                     for (int kb = 0; kb < nkb; ++kb) {
                         if (!mbar_wait(full_bar(stage), phase, abort_flag, args.status, STATUS_WAIT_FULL)) {
                             alive = false; break;
@@ -619,25 +611,14 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                         const uint32_t sA = smem_base + stage * TC_STAGE_BYTES;
                         const uint64_t da = desc_a | (uint64_t)((sA & 0x3ffffu) >> 4);
                         const uint64_t db = desc_b | (uint64_t)(((sA + TC_A_BYTES) & 0x3ffffu) >> 4);
-                        const int kseg = Tr::SEG_KB ? kb % Tr::SEG_KB : kb;   // position inside the accumulation segment
 #pragma unroll
                         for (int k4 = 0; k4 < TC_BK / 16; ++k4)
-                            umma_bf16(d_tmem, da + k4 * 2, db + k4 * b_step, idesc, (kseg | k4) != 0 ? 1u : 0u);
+                            umma_bf16(d_tmem, da + k4 * 2, db + k4 * b_step, idesc, (kb | k4) != 0 ? 1u : 0u);
                         umma_commit(empty_bar(stage));
                         if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
-                        if (Tr::SEG_KB && kseg == Tr::SEG_KB - 1 && kb + 1 < nkb) {
-                            // segment done: hand this accumulator to the epilogue and go on in the other one
-                            umma_commit(tfull_bar(it & 1));
-                            ++it;
-                            const int nb = it & 1;
-                            if (!mbar_wait(tempty_bar(nb), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, args.status,
-                                           STATUS_WAIT_TMEM_EMPTY)) { alive = false; break; }
-                            tc_fence_after();
-                            d_tmem = tmem_base + (uint32_t)nb * TC_BN;
-                        }
                     }
                     if (!alive) break;
-                    umma_commit(tfull_bar(it & 1));
+                    umma_commit(tfull_bar(buf));
                     ++it;
                 }
             }
@@ -723,44 +704,6 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                     }
                     continue;
                 }
-            }
-            if constexpr (KIND == TC_RS) {
-                // Router logits: the K loop arrives in segments, each in a fresh accumulator; this warp adds its
-                // 32 rows x 128 columns of every segment to fp32 registers (round to nearest) and stores at the end.
-                float sum[4][32];
-#pragma unroll
-                for (int g = 0; g < 4; ++g)
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) sum[g][i] = 0.0f;
-                const int nseg = (Tr::PHASES * args.kblocks + Tr::SEG_KB - 1) / Tr::SEG_KB;
-                bool ok = true;
-                for (int sg = 0; sg < nseg; ++sg) {
-                    const int b = it & 1;
-                    if (!mbar_wait_warp(tfull_bar(b), (uint32_t)(it >> 1) & 1u, abort_flag, args.status,
-                                        STATUS_WAIT_TMEM_FULL, lane)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)b * TC_BN + half * 128;
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        float part[32];
-                        tmem_ld32(ta + 32 * g, part);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) sum[g][i] += part[i];
-                    }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar(b));
-                    ++it;
-                }
-                if (!ok) break;
-                if (r < ti.rows) {
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const int col = n0 + half * 128 + 32 * g;
-                        if (col < args.N) epi_f32<32>(args.ep.outf + (size_t)(ti.row0 + r) * args.N + col, sum[g], 0);
-                    }
-                }
-                continue;
             }
             const int buf = it & 1;
             const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
@@ -939,7 +882,6 @@ inline mop_status tc_plan_init(TcPlan* p, const mop_moe_shape& s, int sm_count, 
     if ((r = tc_set_smem<TC_VL>()) != MOP_OK) return r;
     if ((r = tc_set_smem<TC_VP>()) != MOP_OK) return r;
     if ((r = tc_set_smem<TC_VX>()) != MOP_OK) return r;
-    if ((r = tc_set_smem<TC_RS>()) != MOP_OK) return r;
     return MOP_OK;
 }
 

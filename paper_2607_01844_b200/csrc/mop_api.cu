@@ -12,6 +12,7 @@
 #include "epilogue.cuh"
 #include "gemm_scalar.cuh"
 #include "gemm_host.cuh"
+#include "gemm_rs.cuh"
 #include "permute.cuh"
 #include "route.cuh"
 
@@ -41,7 +42,7 @@ struct mop_ctx {
     cudaEvent_t fr_fork, fr_join;
     bf16* fr_pieces;
     float *fr_wrT, *fr_colsq, *fr_xnorm, *fr_scal, *fr_wsq;
-    int32_t *fr_off, *fr_tiles;
+    int32_t* fr_todo;
     // host-buffer entry point scratch
     bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
     int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
@@ -75,7 +76,7 @@ constexpr uint32_t GUARD_PATTERN = 0xA5C3A5C3u;
 
 struct Layout {
     size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT, rG, rU, rH;
-    size_t fr_pieces, fr_wrT, fr_colsq, fr_xnorm, fr_scal, fr_off, fr_tiles, fr_wsq;
+    size_t fr_pieces, fr_wrT, fr_colsq, fr_xnorm, fr_scal, fr_wsq, fr_todo;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
     size_t hG, hU, hdY, hdX, hdgate;
     size_t qx, qY, qidx, qgate, qdY, qdX, qdgate;   // second slot of the pipelined host entry points
@@ -131,8 +132,7 @@ Layout make_layout(const mop_moe_shape& s) {
         L.fr_xnorm = take(T * 4 + 16);
         L.fr_scal = take(256);
         L.fr_wsq = take(E * 4);
-        L.fr_off = take(16);
-        L.fr_tiles = take(tc_tile_table_bytes(s.T, 1));
+        L.fr_todo = take(T * 4 + 16);
     }
     if (s.with_backward) {
         L.part = take((size_t)part_tiles(s) * M * 4);
@@ -317,8 +317,7 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         c->fr_xnorm = reinterpret_cast<float*>(w + L.fr_xnorm);
         c->fr_scal = reinterpret_cast<float*>(w + L.fr_scal);
         c->fr_wsq = reinterpret_cast<float*>(w + L.fr_wsq);
-        c->fr_off = reinterpret_cast<int32_t*>(w + L.fr_off);
-        c->fr_tiles = reinterpret_cast<int32_t*>(w + L.fr_tiles);
+        c->fr_todo = reinterpret_cast<int32_t*>(w + L.fr_todo);
         c->fast_route = route_fast_wanted(*shape);
     } else if (shape->route_path == MOP_ROUTE_TENSOR) {
         cudaFree(c->ws); delete c;
@@ -400,15 +399,10 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         st = tc_plan_init(&c->plan, *shape, c->sm_count, &c->prof);
         if (st == MOP_OK) st = tc2_init();
         if (st == MOP_OK) st = tn_init();
+        if (st == MOP_OK) st = rs_init();
         if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
-        if (c->fast_route) {   // the logit GEMM's row tiles depend on T alone: built once
-            const int32_t host_off[2] = {0, shape->T};
-            bool ok = cudaMemcpy(c->fr_off, host_off, sizeof(host_off), cudaMemcpyHostToDevice) == cudaSuccess &&
-                      cudaMemset(c->fr_scal, 0, 256) == cudaSuccess;
-            if (ok) {
-                tc_build_mtiles_kernel<<<1, 1024>>>(c->fr_off, 1, reinterpret_cast<int4*>(c->fr_tiles + 64), c->fr_tiles);
-                ok = cudaDeviceSynchronize() == cudaSuccess;
-            }
+        if (c->fast_route) {
+            bool ok = cudaMemset(c->fr_scal, 0, 256) == cudaSuccess;
             ok = ok && cudaStreamCreateWithFlags(&c->fr_stream, cudaStreamNonBlocking) == cudaSuccess &&
                  cudaEventCreateWithFlags(&c->fr_fork, cudaEventDisableTiming) == cudaSuccess &&
                  cudaEventCreateWithFlags(&c->fr_join, cudaEventDisableTiming) == cudaSuccess;
@@ -553,22 +547,24 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
                route_prep_kernel<<<gp, 256, 0, st>>>(W_r, c->fr_pieces, c->fr_wrT, c->fr_colsq, s.d, s.E);
                route_wnorm_kernel<<<ceil_div(s.E, 8), 256, 0, st>>>(c->fr_colsq, c->fr_wsq, ceil_div(s.d, 32), s.E));
         if ((r = after_launch(c, 3)) != MOP_OK) return r;
-        CUtensorMap mX, mW;
-        if (!tc_map_2d(&c->plan, &mX, x, s.T, s.d, 128) || !tc_map_chunked_3d(&c->plan, &mW, c->fr_pieces, 3, s.d, s.E, 4))
-            return MOP_ERR_CUDA;
-        TcArgs g{};
-        g.offsets = c->fr_off; g.n_mtiles = c->fr_tiles; g.mtiles = reinterpret_cast<const int4*>(c->fr_tiles + 64);
-        g.E = 1; g.status = c->status;
-        g.tiles_n = ceil_div(s.E, 256); g.kblocks = ceil_div(s.d, TC_BK); g.N = s.E; g.m_fastest = 1;
-        g.ep.outf = z; g.ep.accumulate = 0; g.ep.M_total = s.T;
-        if ((r = tc_launch<TC_RS>(&c->plan, "route_score_tc", mX, mX, mW, mW, mX, mX, g, st)) != MOP_OK) return r;
+        if ((r = rs_launch(&c->plan, "route_score_tc", x, c->fr_pieces, z, s.T, s.d, s.E, c->status, st)) != MOP_OK) return r;
         c->launches += 1;
         CUDA_OK(cudaStreamWaitEvent(st, c->fr_join, 0));
+        int32_t* stats = reinterpret_cast<int32_t*>(c->fr_scal) + 8;
+        int32_t* n_todo = reinterpret_cast<int32_t*>(c->fr_scal) + 16;
+        CUDA_OK(cudaMemsetAsync(n_todo, 0, 4, st));
+        LAUNCH(c, "route_select_screen", st,
+               route_screen_kernel<<<ceil_div(s.T, SCREEN_WARPS), SCREEN_WARPS * 32,
+                                     (size_t)SCREEN_WARPS * 2 * s.E * sizeof(float), st>>>(
+                   z, bias, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate, c->fr_todo, n_todo, s.T, s.d, s.E, s.k, s.score_fn,
+                   s.bias_mode));
+        if ((r = after_launch(c)) != MOP_OK) return r;
         const size_t fsmem = (size_t)SELF_WARPS * (3 * s.E + SELF_SMEM_FLOATS) * sizeof(float);
-        LAUNCH(c, "route_select_fast", st,
-               route_select_fast_kernel<<<ceil_div(s.T, SELF_WARPS), SELF_WARPS * 32, fsmem, st>>>(
-                   z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
-                   reinterpret_cast<int32_t*>(c->fr_scal) + 8, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode));
+        const int rblocks = min(ceil_div(s.T, SELF_WARPS), c->sm_count * 12);
+        LAUNCH(c, "route_select_resolve", st,
+               route_resolve_kernel<<<rblocks, SELF_WARPS * 32, fsmem, st>>>(
+                   z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate, c->fr_todo,
+                   n_todo, stats, s.d, s.E, s.k, s.score_fn, s.bias_mode));
         return after_launch(c);
     }
     LAUNCH(c, "route_score", st, route_score(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E, c->sm_count, st));

@@ -287,8 +287,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) route_select_kernel(const floa
 //
 // 1. W_r (fp32) is split into three bf16 pieces, hi + mid + lo = W_r to 2^-24 relative (each
 //    residual is exact in fp32), and x (bf16) is multiplied by the pieces on the tensor cores: z~
-//    (kind TC_RS of the grouped GEMM; the K loop is summed in segments of 512 so that the truncating
-//    accumulation inside the tensor core stays short, the segments are added in fp32 registers).
+//    (route_score_pair_kernel; the K loop is summed in segments of 192, all three pieces, so that the
+//    truncating accumulation inside the tensor core stays short; the segments are added in fp32 registers).
 //    Every product is exact; what separates z~ from the contract's logit z (one fp32 fused
 //    multiply-add per i, i ascending) is the rounding of the two summations.  Each rounding is at most
 //    u = 2^-24 of a partial sum, and the partial sums of a logit grow like a random walk towards
@@ -427,19 +427,17 @@ __device__ __forceinline__ float key_error(float zz, float ez, int score_fn, int
     return 1.001f * (s * (1.0f - s) + 0.125f * ez) * ez + 4e-7f;         // |s''| <= 0.1; rounding of the sequence
 }
 
-__global__ void __launch_bounds__(SELF_WARPS * 32) route_select_fast_kernel(
-    float* __restrict__ z, const float* __restrict__ bias, const bf16* __restrict__ x, const float* __restrict__ W_rT,
-    const float* __restrict__ xnorm, const float* __restrict__ wsq, int32_t* __restrict__ idx,
-    float* __restrict__ gate, int32_t* __restrict__ stats, int T, int d, int E, int k, int score_fn, int bias_mode) {
-    extern __shared__ float sel_smem[];
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    float* key = sel_smem + (size_t)warp * (3 * E + SELF_SMEM_FLOATS);
-    float* zg = key + E;
-    int32_t* clist = reinterpret_cast<int32_t*>(zg + E);   // experts whose exact logit is needed
-    float* xs = zg + 2 * E;                                 // a chunk of the token's row, fp32
-    float* ws = xs + SELF_XCHUNK;                           // the same chunk of up to SELF_CAND rows of W_r^T
-    const int t = blockIdx.x * SELF_WARPS + warp;
-    if (t >= T) return;
+// One token, one warp.  RESOLVE = false: the screening pass; it returns false, writing nothing, as soon as some
+// order or gate is in doubt.  RESOLVE = true: evaluates the chains in doubt until everything is settled.
+// key, zg: E floats each; clist: E ints, xs, ws: staging of the chains (RESOLVE only).
+template <bool RESOLVE>
+__device__ __forceinline__ bool route_token(int t, int lane, float* key, float* zg, int32_t* clist, float* xs, float* ws,
+                                            float* __restrict__ z, const float* __restrict__ bias,
+                                            const bf16* __restrict__ x, const float* __restrict__ W_rT,
+                                            const float* __restrict__ xnorm, const float* __restrict__ wsq,
+                                            int32_t* __restrict__ idx, float* __restrict__ gate,
+                                            int32_t* __restrict__ stats, int d, int E, int k, int score_fn,
+                                            int bias_mode) {
     float* zrow = z + (size_t)t * E;
     for (int e = lane; e < E; e += 32) {
         float zz = zrow[e];
@@ -488,6 +486,7 @@ __global__ void __launch_bounds__(SELF_WARPS * 32) route_select_fast_kernel(
             }
             const uint32_t m = __ballot_sync(0xffffffffu, cand);
             if (m) {
+                if constexpr (!RESOLVE) return false;
                 if (cand) clist[n_c + __popc(m & ((1u << lane) - 1u))] = e;
                 n_c += __popc(m);
             }
@@ -503,6 +502,10 @@ __global__ void __launch_bounds__(SELF_WARPS * 32) route_select_fast_kernel(
         // picks in doubt whose logit is still approximate join the list
         const bool need = doubt && !pick_exact;
         const uint32_t m = __ballot_sync(0xffffffffu, need);
+        if constexpr (!RESOLVE) {
+            if (m) return false;
+            break;
+        }
         if (need) clist[n_c + __popc(m & ((1u << lane) - 1u))] = my_e;
         n_c += __popc(m);
         if (n_c == 0) break;                         // every order that matters is settled (exact ties go by id)
@@ -575,7 +578,7 @@ __global__ void __launch_bounds__(SELF_WARPS * 32) route_select_fast_kernel(
         n_chains += n_c;
         __syncwarp();
     }
-    if (stats && n_chains > 0) {                     // statistics only: no result depends on them
+    if (RESOLVE && stats && n_chains > 0) {          // statistics only: no result depends on them
         n_bad = __reduce_add_sync(0xffffffffu, n_bad);
         if (lane == 0) { atomicAdd(stats, 1); atomicAdd(stats + 1, n_chains); if (n_bad) atomicAdd(stats + 2, n_bad); }
     }
@@ -595,6 +598,46 @@ __global__ void __launch_bounds__(SELF_WARPS * 32) route_select_fast_kernel(
     if (act) {
         idx[(size_t)t * k + lane] = my_e;
         gate[(size_t)t * k + lane] = s / sum;
+    }
+    return true;
+}
+
+// Screening pass: every token, one warp each, little shared memory (high occupancy).  Tokens whose approximate
+// keys settle everything are finished here; the others are listed for the resolving pass.  The list's order
+// depends on timing, no result does.
+constexpr int SCREEN_WARPS = 4;
+__global__ void __launch_bounds__(SCREEN_WARPS * 32) route_screen_kernel(
+    float* __restrict__ z, const float* __restrict__ bias, const float* __restrict__ xnorm,
+    const float* __restrict__ wsq, int32_t* __restrict__ idx, float* __restrict__ gate, int32_t* __restrict__ todo,
+    int32_t* __restrict__ n_todo, int T, int d, int E, int k, int score_fn, int bias_mode) {
+    extern __shared__ float sel_smem[];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    float* key = sel_smem + (size_t)warp * 2 * E;
+    const int t = blockIdx.x * SCREEN_WARPS + warp;
+    if (t >= T) return;
+    const bool done = route_token<false>(t, lane, key, key + E, nullptr, nullptr, nullptr, z, bias, nullptr, nullptr, xnorm,
+                                         wsq, idx, gate, nullptr, d, E, k, score_fn, bias_mode);
+    if (!done && lane == 0) todo[atomicAdd(n_todo, 1)] = t;
+}
+
+// Resolving pass: the listed tokens, one warp each, with the staging memory of the chains.
+__global__ void __launch_bounds__(SELF_WARPS * 32) route_resolve_kernel(
+    float* __restrict__ z, const float* __restrict__ bias, const bf16* __restrict__ x, const float* __restrict__ W_rT,
+    const float* __restrict__ xnorm, const float* __restrict__ wsq, int32_t* __restrict__ idx,
+    float* __restrict__ gate, const int32_t* __restrict__ todo, const int32_t* __restrict__ n_todo,
+    int32_t* __restrict__ stats, int d, int E, int k, int score_fn, int bias_mode) {
+    extern __shared__ float sel_smem[];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    float* key = sel_smem + (size_t)warp * (3 * E + SELF_SMEM_FLOATS);
+    float* zg = key + E;
+    int32_t* clist = reinterpret_cast<int32_t*>(zg + E);   // experts whose exact logit is needed
+    float* xs = zg + 2 * E;                                 // a chunk of the token's row, fp32
+    float* ws = xs + SELF_XCHUNK;                           // the same chunk of up to SELF_CAND rows of W_r^T
+    const int n = *n_todo;
+    for (int i = blockIdx.x * SELF_WARPS + warp; i < n; i += gridDim.x * SELF_WARPS) {
+        route_token<true>(todo[i], lane, key, zg, clist, xs, ws, z, bias, x, W_rT, xnorm, wsq, idx, gate, stats, d, E, k,
+                          score_fn, bias_mode);
+        __syncwarp();
     }
 }
 
