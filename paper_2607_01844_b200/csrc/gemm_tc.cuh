@@ -726,7 +726,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                 // the four warps of a column half stage 128 rows x 32 fp32 columns in shared memory (128-byte
                 // rows, 16-byte chunks XOR-swizzled by row: the layout of a 128B-swizzle tensor map,
                 // conflict-free for one-row-per-lane writes) and one thread hands the 16 KiB box to TMA, which
-                // writes whole 128-byte lines and clips rows >= Mfix and columns >= N.  Two boxes per half.
+                // writes whole 128-byte lines and clips rows >= Mfix and columns >= N.  Two boxes per half: one
+                // is being read by the copy engine while the next one is staged.
                 uint8_t* gbase = smem + TC_STAGES * TC_STAGE_BYTES + TC_BAR_BYTES + half * 32768;
                 const CUtensorMap* mo = (Tr::SEL_B && ti.sel) ? &tmO1 : &tmO0;
                 const bool issuer = (quarter == 0 && lane == 0);
@@ -744,8 +745,6 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     uint8_t* box = gbase + (sbuf & 1) * 16384;
-                    if (issuer) tma_store_wait_read<1>();     // the box staged two steps ago has been read
-                    asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
                     uint8_t* rowp = box + (quarter * 32 + lane) * 128;
                     const float(&v)[32] = cc == 0 ? a0 : cc == 1 ? a1 : cc == 2 ? a2 : a3;
 #pragma unroll
@@ -753,6 +752,9 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_co
                         *reinterpret_cast<float4*>(rowp + ((j ^ (lane & 7)) << 4)) =
                             make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    // One barrier per step.  Before it the issuing thread makes sure that the box handed over one
+                    // step ago has been read, so after it everyone may overwrite that box (the next step's).
+                    if (issuer) tma_store_wait_read<0>();
                     asm volatile("bar.sync %0, 128;" ::"r"(gbar) : "memory");
                     if (issuer) {
                         const int gcol = n0 + half * 128 + 32 * cc;

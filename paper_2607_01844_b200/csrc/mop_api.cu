@@ -553,18 +553,14 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
         int32_t* stats = reinterpret_cast<int32_t*>(c->fr_scal) + 8;
         int32_t* n_todo = reinterpret_cast<int32_t*>(c->fr_scal) + 16;
         CUDA_OK(cudaMemsetAsync(n_todo, 0, 4, st));
-        LAUNCH(c, "route_select_screen", st,
-               route_screen_kernel<<<ceil_div(s.T, SCREEN_WARPS), SCREEN_WARPS * 32,
-                                     (size_t)SCREEN_WARPS * 2 * s.E * sizeof(float), st>>>(
-                   z, bias, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate, c->fr_todo, n_todo, s.T, s.d, s.E, s.k, s.score_fn,
-                   s.bias_mode));
-        if ((r = after_launch(c)) != MOP_OK) return r;
-        const size_t fsmem = (size_t)SELF_WARPS * (3 * s.E + SELF_SMEM_FLOATS) * sizeof(float);
         const int rblocks = min(ceil_div(s.T, SELF_WARPS), c->sm_count * 12);
+        LAUNCH(c, "route_select_screen", st,
+               route_select_fast(z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
+                                 c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 0, rblocks, st));
+        if ((r = after_launch(c)) != MOP_OK) return r;
         LAUNCH(c, "route_select_resolve", st,
-               route_resolve_kernel<<<rblocks, SELF_WARPS * 32, fsmem, st>>>(
-                   z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate, c->fr_todo,
-                   n_todo, stats, s.d, s.E, s.k, s.score_fn, s.bias_mode));
+               route_select_fast(z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
+                                 c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 1, rblocks, st));
         return after_launch(c);
     }
     LAUNCH(c, "route_score", st, route_score(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E, c->sm_count, st));

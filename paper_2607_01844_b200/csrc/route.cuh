@@ -388,81 +388,104 @@ constexpr float ROUTE_GATE_REL = 5e-6f;   // a pick whose gate could be off by m
 constexpr int SELF_XCHUNK = 256;  // elements of the token's row staged per step of the exact chains
 constexpr int SELF_CAND = 4;      // chains evaluated side by side (one lane each), their W_r^T rows staged in shared memory
 constexpr int SELF_WPITCH = SELF_XCHUNK + 4;   // row pitch of the staged W_r^T chunks: lanes read different banks
-constexpr int SELF_SMEM_FLOATS = SELF_XCHUNK + SELF_CAND * SELF_WPITCH;   // per warp, besides the 3 E key / logit / list words
+constexpr int SELF_SMEM_FLOATS = SELF_XCHUNK + SELF_CAND * SELF_WPITCH;   // per warp, besides the 2 E logit / list words
 
-// k selection rounds over the keys in shared memory (as in route_select_kernel).  Lane j < k keeps the j-th
-// pick: its expert, its key and the logit its gate is computed from; `taken` marks this lane's picked experts.
-__device__ __forceinline__ void select_rounds(const float* key, const float* zg, int E, int k, int lane, int& my_e,
-                                              float& my_key, float& my_z, uint32_t& taken) {
+// Order-preserving map of a finite float to an unsigned integer (-0 counts as +0, as in a float comparison).
+__device__ __forceinline__ uint32_t key_ord(float f) {
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// k selection rounds over keys held in registers: lane l owns the experts e = l + 32 q, q < Q, key kv[q].
+// A round is two warp reductions (largest key among the lanes' best untaken keys, then the lowest expert id
+// among the lanes that hold it) and a rescan of the winner's own keys.  Lane j < k keeps the j-th pick: its
+// expert, its key and the logit its gate is computed from; `taken` marks this lane's picked experts.
+// Same order as route_select_kernel: larger key first, equal keys by lower id.
+template <int Q>
+__device__ __forceinline__ void select_rounds_reg(const float (&kv)[Q], uint32_t invalid, const float* zg, int k, int lane,
+                                                  int& my_e, float& my_key, float& my_z, uint32_t& taken) {
     taken = 0;
     my_e = -1; my_key = 0.0f; my_z = 0.0f;
-    for (int j = 0; j < k; ++j) {
-        int best = -1;
-        float bk = 0.0f;
-        for (int q = 0, e = lane; e < E; ++q, e += 32) {
-            if ((taken >> q) & 1u) continue;
-            const float v = key[e];
-            if (best < 0 || v > bk) { best = e; bk = v; }
-        }
+    float bk = 0.0f; int bq = -1;
+    auto rescan = [&]() {
+        bq = -1; bk = 0.0f;
+        const uint32_t off = taken | invalid;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ok = __shfl_xor_sync(0xffffffffu, bk, off);
-            const int oe = __shfl_xor_sync(0xffffffffu, best, off);
-            const bool take = (oe >= 0) && (best < 0 || ok > bk || (ok == bk && oe < best));
-            if (take) { bk = ok; best = oe; }
-        }
-        if ((best & 31) == lane) taken |= 1u << (best >> 5);
-        if (j == lane) { my_e = best; my_key = bk; my_z = zg[best]; }
+        for (int q = 0; q < Q; ++q)
+            if (!((off >> q) & 1u) && (bq < 0 || kv[q] > bk)) { bq = q; bk = kv[q]; }
+    };
+    rescan();
+    for (int j = 0; j < k; ++j) {
+        const uint32_t mine = bq >= 0 ? key_ord(bk) : 0u;            // 0 lies below the image of every finite key
+        const uint32_t top = __reduce_max_sync(0xffffffffu, mine);
+        const int cand = (bq >= 0 && mine == top) ? lane + 32 * bq : 0x7fffffff;
+        const int win = __reduce_min_sync(0xffffffffu, cand);
+        const float wkey = __shfl_sync(0xffffffffu, bk, win & 31);
+        if ((win & 31) == lane) { taken |= 1u << (win >> 5); rescan(); }
+        if (j == lane) { my_e = win; my_key = wkey; my_z = zg[win]; }
     }
 }
 
 __device__ __forceinline__ float route_key(float zz, float b, int score_fn, int bias_mode) {
     return (score_fn == 1 && bias_mode == 1) ? __fadd_rn(sigmoid_contract(zz), b) : zz;
 }
+// Key of an approximate logit: the sigmoid by the fast exponential and division.  Against the contract's sequence it is
+// off by less than 1e-6 (exponential: 2 + 1.173 |z| ulp, times the slope s (1 - s): at most 8e-8; division 2 ulp;
+// the contract's own polynomial 2e-7), which key_error adds to the interval of such a key.
+constexpr float ROUTE_FAST_KEY_ERR = 1e-6f;
+__device__ __forceinline__ float route_key_approx(float zz, float b, int score_fn, int bias_mode) {
+    return (score_fn == 1 && bias_mode == 1) ? sigmoidf_fast(zz) + b : zz;
+}
 
-// Bound on the error of a key whose logit is off by at most ez (a little slack covers its own rounding).
+// Bound on the error of an approximate key whose logit is off by at most ez (a little slack covers its own rounding).
 __device__ __forceinline__ float key_error(float zz, float ez, int score_fn, int bias_mode) {
     if (!(score_fn == 1 && bias_mode == 1)) return ez;                   // the key is the logit itself
-    const float s = sigmoidf_acc(zz);
-    return 1.001f * (s * (1.0f - s) + 0.125f * ez) * ez + 4e-7f;         // |s''| <= 0.1; rounding of the sequence
+    const float s = sigmoidf_fast(zz);
+    return 1.001f * (s * (1.0f - s) + 0.125f * ez) * ez + 4e-7f + ROUTE_FAST_KEY_ERR;   // |s''| <= 0.1
 }
 
 // One token, one warp.  RESOLVE = false: the screening pass; it returns false, writing nothing, as soon as some
 // order or gate is in doubt.  RESOLVE = true: evaluates the chains in doubt until everything is settled.
-// key, zg: E floats each; clist: E ints, xs, ws: staging of the chains (RESOLVE only).
-template <bool RESOLVE>
-__device__ __forceinline__ bool route_token(int t, int lane, float* key, float* zg, int32_t* clist, float* xs, float* ws,
+// Lane l holds the keys of the experts l + 32 q in registers (Q = ceil(E / 32) rounded up to a supported size).
+// zg: E floats (logits); clist: E ints, xs, ws: staging of the chains (RESOLVE only).
+template <bool RESOLVE, int Q>
+__device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t* clist, float* xs, float* ws,
                                             float* __restrict__ z, const float* __restrict__ bias,
                                             const bf16* __restrict__ x, const float* __restrict__ W_rT,
-                                            const float* __restrict__ xnorm, const float* __restrict__ wsq,
-                                            int32_t* __restrict__ idx, float* __restrict__ gate,
-                                            int32_t* __restrict__ stats, int d, int E, int k, int score_fn,
-                                            int bias_mode) {
+                                            const float* __restrict__ xnorm, float wmax, int32_t* __restrict__ idx,
+                                            float* __restrict__ gate, int32_t* __restrict__ stats, int d, int E, int k,
+                                            int score_fn, int bias_mode) {
     float* zrow = z + (size_t)t * E;
-    for (int e = lane; e < E; e += 32) {
-        float zz = zrow[e];
-        const float b = bias_mode ? bias[e] : 0.0f;
-        if (bias_mode == 2) zz = __fadd_rn(zz, b);
-        key[e] = route_key(zz, b, score_fn, bias_mode);
-        zg[e] = zz;
+    float kv[Q];
+    uint32_t invalid = 0;                            // slots q of this lane beyond E
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+        const int e = lane + 32 * q;
+        kv[q] = 0.0f;
+        if (e < E) {
+            float zz = zrow[e];
+            const float b = bias_mode ? bias[e] : 0.0f;
+            if (bias_mode == 2) zz = __fadd_rn(zz, b);
+            kv[q] = route_key_approx(zz, b, score_fn, bias_mode);
+            zg[e] = zz;
+        } else {
+            invalid |= 1u << q;
+        }
     }
     __syncwarp();
     // Bound of this token's logit error (see above).
-    float wmax2 = 0.0f;                              // largest squared column norm of W_r
-    for (int e = lane; e < E; e += 32) wmax2 = fmaxf(wmax2, wsq[e]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) wmax2 = fmaxf(wmax2, __shfl_xor_sync(0xffffffffu, wmax2, off));
-    const float scale = 5.9604645e-8f * xnorm[t] * sqrtf(wmax2);
+    const float scale = 5.9604645e-8f * xnorm[t] * wmax;
     const float ez = ROUTE_EPS_C * scale, ez_gate = ROUTE_EPS_GATE_C * scale;
-    uint32_t exact = 0;                              // this lane's experts (e = lane + 32 q) that carry the chain's logit
+    uint32_t exact = 0;                              // this lane's experts that carry the chain's logit
     int my_e; float my_key, my_z; uint32_t taken;
     int n_chains = 0, n_bad = 0;
     for (int iter = 0; iter <= k + 1; ++iter) {
-        select_rounds(key, zg, E, k, lane, my_e, my_key, my_z, taken);
+        select_rounds_reg<Q>(kv, invalid, zg, k, lane, my_e, my_key, my_z, taken);
         // interval [lo, hi] that holds the exact key of each pick (a point once the chain was evaluated)
         const bool pick = lane < k;
-        const uint32_t pick_exact = pick ? (__shfl_sync(0xffffffffu, exact, my_e & 31) >> (my_e >> 5)) & 1u
-                                         : (__shfl_sync(0xffffffffu, exact, 0), 1u);
+        const uint32_t owner_exact = __shfl_sync(0xffffffffu, exact, pick ? (my_e & 31) : 0);
+        const uint32_t pick_exact = pick ? (owner_exact >> (my_e >> 5)) & 1u : 1u;
         const float my_err = (pick && !pick_exact) ? key_error(my_z, ez, score_fn, bias_mode) : 0.0f;
         const float lo = pick ? my_key - my_err : INFINITY, hi = pick ? my_key + my_err : -INFINITY;
         const float next_hi = __shfl_down_sync(0xffffffffu, hi, 1), prev_lo = __shfl_up_sync(0xffffffffu, lo, 1);
@@ -473,30 +496,39 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* key, float* 
         for (int off = 16; off > 0; off >>= 1) lo_min = fminf(lo_min, __shfl_xor_sync(0xffffffffu, lo_min, off));
         // outsiders that could reach the weakest pick, and the picks they could reach.  Nearly all of them
         // fail already with the largest error any key can have (slope 1/4), which costs no transcendental.
-        const float err_any = (score_fn == 1 && bias_mode == 1) ? 1.001f * (0.25f + 0.125f * ez) * ez + 4e-7f : ez;
+        const float err_any = (score_fn == 1 && bias_mode == 1)
+                                  ? 1.001f * (0.25f + 0.125f * ez) * ez + 4e-7f + ROUTE_FAST_KEY_ERR : ez;
         float out_hi = -INFINITY;
         int n_c = 0;
-        for (int e0 = 0; e0 < E; e0 += 32) {
-            const int e = e0 + lane, q = e0 >> 5;
+        bool any_cand = false;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const int e = lane + 32 * q;
             bool cand = false;
-            if (e < E && !((taken >> q) & 1u) && !(key[e] + err_any < lo_min)) {
+            if (!(((taken | invalid) >> q) & 1u) && !(kv[q] + err_any < lo_min)) {
                 const bool ex = (exact >> q) & 1u;
-                const float h = key[e] + (ex ? 0.0f : key_error(zg[e], ez, score_fn, bias_mode));
+                const float h = kv[q] + (ex ? 0.0f : key_error(zg[e], ez, score_fn, bias_mode));
                 if (!(h < lo_min)) { out_hi = fmaxf(out_hi, h); cand = !ex; }
             }
-            const uint32_t m = __ballot_sync(0xffffffffu, cand);
-            if (m) {
-                if constexpr (!RESOLVE) return false;
-                if (cand) clist[n_c + __popc(m & ((1u << lane) - 1u))] = e;
-                n_c += __popc(m);
+            if constexpr (RESOLVE) {
+                const uint32_t m = __ballot_sync(0xffffffffu, cand);
+                if (m) {
+                    if (cand) clist[n_c + __popc(m & ((1u << lane) - 1u))] = e;
+                    n_c += __popc(m);
+                }
+            } else {
+                any_cand |= cand;
             }
+        }
+        if constexpr (!RESOLVE) {
+            if (__any_sync(0xffffffffu, any_cand)) return false;
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) out_hi = fmaxf(out_hi, __shfl_xor_sync(0xffffffffu, out_hi, off));
         if (pick && !(lo > out_hi)) doubt = true;
         // gates: d g / g = (1 - s) dz for a sigmoid score, at most dz for a softmax over the picks
         if (pick && !pick_exact) {
-            const float sens = (score_fn == 1) ? 1.0f - sigmoidf_acc(my_z) : 1.0f;
+            const float sens = (score_fn == 1) ? 1.0f - sigmoidf_fast(my_z) : 1.0f;
             if (sens * ez_gate > ROUTE_GATE_REL) doubt = true;
         }
         // picks in doubt whose logit is still approximate join the list
@@ -561,18 +593,25 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* key, float* 
                     }
                 }
             }
+            float newkey = 0.0f;
             if (mine) {
                 if (fabsf(zrow[e] - acc) > 0.5f * ez) ++n_bad;       // the model of the error is checked as we go
                 zrow[e] = acc;                       // the exact logit replaces the approximate one
                 const float b = bias_mode ? bias[e] : 0.0f;
                 const float zz = (bias_mode == 2) ? __fadd_rn(acc, b) : acc;
-                key[e] = route_key(zz, b, score_fn, bias_mode);
+                newkey = route_key(zz, b, score_fn, bias_mode);      // the contract's key
                 zg[e] = zz;
             }
-            // mark the evaluated experts in their owner lanes' masks
+            // the evaluated experts' keys go to their owner lanes, which mark them exact
             for (int j = 0; j < nc; ++j) {
                 const int ej = clist[c0 + j];
-                if ((ej & 31) == lane) exact |= 1u << (ej >> 5);
+                const float kj = __shfl_sync(0xffffffffu, newkey, j);
+                if ((ej & 31) == lane) {
+                    exact |= 1u << (ej >> 5);
+#pragma unroll
+                    for (int q = 0; q < Q; ++q)
+                        if (q == (ej >> 5)) kv[q] = kj;
+                }
             }
         }
         n_chains += n_c;
@@ -602,25 +641,36 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* key, float* 
     return true;
 }
 
+// Largest column norm of W_r, from the squared norms: every lane returns it.
+__device__ __forceinline__ float route_wmax(const float* __restrict__ wsq, int E, int lane) {
+    float wmax2 = 0.0f;
+    for (int e = lane; e < E; e += 32) wmax2 = fmaxf(wmax2, wsq[e]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) wmax2 = fmaxf(wmax2, __shfl_xor_sync(0xffffffffu, wmax2, off));
+    return sqrtf(wmax2);
+}
+
 // Screening pass: every token, one warp each, little shared memory (high occupancy).  Tokens whose approximate
 // keys settle everything are finished here; the others are listed for the resolving pass.  The list's order
 // depends on timing, no result does.
 constexpr int SCREEN_WARPS = 4;
+template <int Q>
 __global__ void __launch_bounds__(SCREEN_WARPS * 32) route_screen_kernel(
     float* __restrict__ z, const float* __restrict__ bias, const float* __restrict__ xnorm,
     const float* __restrict__ wsq, int32_t* __restrict__ idx, float* __restrict__ gate, int32_t* __restrict__ todo,
     int32_t* __restrict__ n_todo, int T, int d, int E, int k, int score_fn, int bias_mode) {
     extern __shared__ float sel_smem[];
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    float* key = sel_smem + (size_t)warp * 2 * E;
     const int t = blockIdx.x * SCREEN_WARPS + warp;
     if (t >= T) return;
-    const bool done = route_token<false>(t, lane, key, key + E, nullptr, nullptr, nullptr, z, bias, nullptr, nullptr, xnorm,
-                                         wsq, idx, gate, nullptr, d, E, k, score_fn, bias_mode);
+    const float wmax = route_wmax(wsq, E, lane);
+    const bool done = route_token<false, Q>(t, lane, sel_smem + (size_t)warp * E, nullptr, nullptr, nullptr, z, bias, nullptr,
+                                            nullptr, xnorm, wmax, idx, gate, nullptr, d, E, k, score_fn, bias_mode);
     if (!done && lane == 0) todo[atomicAdd(n_todo, 1)] = t;
 }
 
 // Resolving pass: the listed tokens, one warp each, with the staging memory of the chains.
+template <int Q>
 __global__ void __launch_bounds__(SELF_WARPS * 32) route_resolve_kernel(
     float* __restrict__ z, const float* __restrict__ bias, const bf16* __restrict__ x, const float* __restrict__ W_rT,
     const float* __restrict__ xnorm, const float* __restrict__ wsq, int32_t* __restrict__ idx,
@@ -628,17 +678,50 @@ __global__ void __launch_bounds__(SELF_WARPS * 32) route_resolve_kernel(
     int32_t* __restrict__ stats, int d, int E, int k, int score_fn, int bias_mode) {
     extern __shared__ float sel_smem[];
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    float* key = sel_smem + (size_t)warp * (3 * E + SELF_SMEM_FLOATS);
-    float* zg = key + E;
+    const int n = *n_todo;
+    if ((int)blockIdx.x * SELF_WARPS >= n) return;
+    float* zg = sel_smem + (size_t)warp * (2 * E + SELF_SMEM_FLOATS);
     int32_t* clist = reinterpret_cast<int32_t*>(zg + E);   // experts whose exact logit is needed
     float* xs = zg + 2 * E;                                 // a chunk of the token's row, fp32
     float* ws = xs + SELF_XCHUNK;                           // the same chunk of up to SELF_CAND rows of W_r^T
-    const int n = *n_todo;
+    const float wmax = route_wmax(wsq, E, lane);
     for (int i = blockIdx.x * SELF_WARPS + warp; i < n; i += gridDim.x * SELF_WARPS) {
-        route_token<true>(todo[i], lane, key, zg, clist, xs, ws, z, bias, x, W_rT, xnorm, wsq, idx, gate, stats, d, E, k,
-                          score_fn, bias_mode);
+        route_token<true, Q>(todo[i], lane, zg, clist, xs, ws, z, bias, x, W_rT, xnorm, wmax, idx, gate, stats, d, E, k,
+                             score_fn, bias_mode);
         __syncwarp();
     }
+}
+
+// The two passes for the smallest supported Q >= ceil(E / 32).
+template <int Q>
+inline void route_select_fast_q(float* z, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
+                                const float* wsq, int32_t* idx, float* gate, int32_t* todo, int32_t* n_todo,
+                                int32_t* stats, int T, int d, int E, int k, int score_fn, int bias_mode, int pass,
+                                int resolve_blocks, cudaStream_t st) {
+    if (pass == 0) {
+        route_screen_kernel<Q><<<ceil_div(T, SCREEN_WARPS), SCREEN_WARPS * 32, (size_t)SCREEN_WARPS * E * sizeof(float), st>>>(
+            z, bias, xnorm, wsq, idx, gate, todo, n_todo, T, d, E, k, score_fn, bias_mode);
+    } else {
+        const size_t smem = (size_t)SELF_WARPS * (2 * E + SELF_SMEM_FLOATS) * sizeof(float);
+        route_resolve_kernel<Q><<<resolve_blocks, SELF_WARPS * 32, smem, st>>>(z, bias, x, W_rT, xnorm, wsq, idx, gate, todo,
+                                                                                n_todo, stats, d, E, k, score_fn, bias_mode);
+    }
+}
+inline void route_select_fast(float* z, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
+                              const float* wsq, int32_t* idx, float* gate, int32_t* todo, int32_t* n_todo, int32_t* stats,
+                              int T, int d, int E, int k, int score_fn, int bias_mode, int pass, int resolve_blocks,
+                              cudaStream_t st) {
+    const int q = ceil_div(E, 32);
+#define MOP_ROUTE_Q(QQ)                                                                                                 \
+    route_select_fast_q<QQ>(z, bias, x, W_rT, xnorm, wsq, idx, gate, todo, n_todo, stats, T, d, E, k, score_fn, bias_mode, \
+                            pass, resolve_blocks, st)
+    if (q <= 2) MOP_ROUTE_Q(2);
+    else if (q <= 4) MOP_ROUTE_Q(4);
+    else if (q <= 8) MOP_ROUTE_Q(8);
+    else if (q <= 12) MOP_ROUTE_Q(12);
+    else if (q <= 16) MOP_ROUTE_Q(16);
+    else MOP_ROUTE_Q(32);
+#undef MOP_ROUTE_Q
 }
 
 // ---------------------------------------------------------------------------------------------
