@@ -39,7 +39,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # (kernel, workload).  Filled from the summaries under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES: dict = {
     # profiles/dram_traffic_gemm_kernels.md: one-pass captures of the full-size launches
-    ("gemm_wgrad_gate_up", "c5_train"): 1477450496 + 45033558528,
+    ("gemm_wgrad_gate_up", "c5_train"): 1477344768 + 45034986752,
     ("gemm_up_swiglu", "c3_trillion"): 24036303104 + 537853952,
     ("gemm_up_swiglu", "c4_skew"): 28745956608 + 538783744,
 }
