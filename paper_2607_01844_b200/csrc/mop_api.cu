@@ -620,10 +620,9 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
                                                                                         row_src, M, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
     if (!Xp) return MOP_OK;
-    const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
     LAUNCH(c, "permute_scatter_rows", st,
-           scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row,
-                                                       s.T, s.k, s.d / 8));
+           launch_scatter_rows(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, s.T, s.k, s.d / 8,
+                               c->sm_count, st));
     return after_launch(c);
 }
 
@@ -634,11 +633,10 @@ mop_status mop_moe_combine(mop_ctx* c, const void* Yp, const int32_t* perm_row, 
     if (s.T == 0) return MOP_OK;
     DeviceGuard guard(c->device);
     if (!guard.ok) return MOP_ERR_CUDA;
-    const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     LAUNCH(c, "combine_rows", st,
-           combine_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(Yp), perm_row, static_cast<uint4*>(Y),
-                                                       s.T, s.k, s.d / 8));
+           launch_combine_rows(static_cast<const uint4*>(Yp), perm_row, static_cast<uint4*>(Y), s.T, s.k, s.d / 8,
+                               c->sm_count, st));
     return after_launch(c);
 }
 
@@ -762,11 +760,9 @@ mop_status mop_moe_expert_ffn_bwd(mop_ctx* c, const void* dY, const void* Xp, co
     }
     if (s.T > 0) {
         // dYp[p,:] = dY[t,:]  (unscaled; the gate enters through dH and gate*H)
-        const int blocks = min(ceil_div(s.T, 8), c->sm_count * 8);
         LAUNCH(c, "dy_scatter_rows", st,
-               scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(dY),
-                                                           reinterpret_cast<uint4*>(c->dYp), perm_row, s.T, s.k,
-                                                           s.d / 8));
+               launch_scatter_rows(static_cast<const uint4*>(dY), reinterpret_cast<uint4*>(c->dYp), perm_row, s.T, s.k,
+                                   s.d / 8, c->sm_count, st));
         if ((r = after_launch(c)) != MOP_OK) return r;
     }
     int ntile_part = 0;
@@ -1355,9 +1351,7 @@ mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, i
                                                                                 M, E);
     if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
     if (!Xp) return MOP_OK;
-    const int blocks = min(ceil_div(T, 8), su.sm_count * 8);
-    scatter_rows_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, T, k,
-                                                d / 8);
+    launch_scatter_rows(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, T, k, d / 8, su.sm_count, st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 

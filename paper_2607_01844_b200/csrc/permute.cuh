@@ -183,6 +183,123 @@ __global__ void __launch_bounds__(256) combine_rows_kernel(const uint4* __restri
     }
 }
 
+// Scatter rows with the whole source row in registers (VPL 16-byte vectors per lane, rows of up to 512 VPL
+// bytes): the row is read once and each of its k copies is written as one contiguous run, which DRAM takes
+// better than pieces of 2 KiB interleaved over k rows (random 2 KiB pieces: 4.4 TB/s at T = 16384, d = 7168).
+template <int VPL>
+__global__ void __launch_bounds__(256) scatter_rows_reg_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
+                                                               const int32_t* __restrict__ perm_row, int T, int k,
+                                                               int vec_per_row) {
+    const int warps_per_block = blockDim.x / 32;
+    const int lane = threadIdx.x % 32;
+    for (int t = blockIdx.x * warps_per_block + threadIdx.x / 32; t < T; t += gridDim.x * warps_per_block) {
+        int32_t myrow = -1;
+        if (lane < k) myrow = perm_row[(size_t)t * k + lane];  // k <= 32 checked on the host
+        const uint4* s = src + (size_t)t * vec_per_row;
+        uint4 v[VPL];
+#pragma unroll
+        for (int q = 0; q < VPL; ++q) {
+            const int c = q * 32 + lane;
+            if (c < vec_per_row) v[q] = __ldg(s + c);
+        }
+        for (int j = 0; j < k; ++j) {
+            const int32_t p = __shfl_sync(0xffffffffu, myrow, j);
+            if (p < 0) continue;
+            uint4* o = dst + (size_t)p * vec_per_row;
+#pragma unroll
+            for (int q = 0; q < VPL; ++q) {
+                const int c = q * 32 + lane;
+                if (c < vec_per_row) __stcs(o + c, v[q]);
+            }
+        }
+    }
+}
+
+// Combine with longer runs per row: the row is walked in segments of 32 SEG vectors (3.5 or 4 KiB); for every
+// segment the k rows are read one after the other, the next row's vectors in flight while the current ones are
+// added.  Same sums in the same order as combine_rows_kernel (j ascending, fp32), so the same bits.
+template <int SEG>
+__global__ void __launch_bounds__(256) combine_rows_seg_kernel(const uint4* __restrict__ Yp,
+                                                               const int32_t* __restrict__ perm_row,
+                                                               uint4* __restrict__ Y, int T, int k, int vec_per_row) {
+    const int warps_per_block = blockDim.x / 32;
+    const int lane = threadIdx.x % 32;
+    for (int t = blockIdx.x * warps_per_block + threadIdx.x / 32; t < T; t += gridDim.x * warps_per_block) {
+        int32_t myrow = -1;
+        if (lane < k) myrow = perm_row[(size_t)t * k + lane];
+        for (int c0 = 0; c0 < vec_per_row; c0 += 32 * SEG) {
+            float acc[SEG][8];
+#pragma unroll
+            for (int q = 0; q < SEG; ++q)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[q][i] = 0.0f;
+            uint4 a[SEG], b[SEG];
+            auto load = [&](uint4 (&buf)[SEG], int j) -> bool {
+                const int32_t p = __shfl_sync(0xffffffffu, myrow, j);
+                if (p < 0) return false;
+                const uint4* r = Yp + (size_t)p * vec_per_row + c0 + lane;
+#pragma unroll
+                for (int q = 0; q < SEG; ++q)
+                    if (c0 + q * 32 + lane < vec_per_row) buf[q] = __ldcs(r + q * 32);
+                return true;
+            };
+            auto add = [&](const uint4 (&buf)[SEG]) {
+#pragma unroll
+                for (int q = 0; q < SEG; ++q) {
+                    if (c0 + q * 32 + lane < vec_per_row) {
+                        const uint4 v = buf[q];
+                        acc[q][0] += bf16_lo(v.x); acc[q][1] += bf16_hi(v.x);
+                        acc[q][2] += bf16_lo(v.y); acc[q][3] += bf16_hi(v.y);
+                        acc[q][4] += bf16_lo(v.z); acc[q][5] += bf16_hi(v.z);
+                        acc[q][6] += bf16_lo(v.w); acc[q][7] += bf16_hi(v.w);
+                    }
+                }
+            };
+            bool va = load(a, 0), vb = false;
+            for (int j = 0; j < k; j += 2) {
+                if (j + 1 < k) vb = load(b, j + 1);
+                if (va) add(a);
+                if (j + 2 < k) va = load(a, j + 2);
+                if (j + 1 < k && vb) add(b);
+            }
+#pragma unroll
+            for (int q = 0; q < SEG; ++q) {
+                const int c = c0 + q * 32 + lane;
+                if (c < vec_per_row) {
+                    uint4 o;
+                    o.x = pack_bf16x2(acc[q][0], acc[q][1]);
+                    o.y = pack_bf16x2(acc[q][2], acc[q][3]);
+                    o.z = pack_bf16x2(acc[q][4], acc[q][5]);
+                    o.w = pack_bf16x2(acc[q][6], acc[q][7]);
+                    Y[(size_t)t * vec_per_row + c] = o;
+                }
+            }
+        }
+    }
+}
+
+// Launchers: the register-row forms for rows of up to 16 KiB, the chunked kernels otherwise.
+inline void launch_scatter_rows(const uint4* src, uint4* dst, const int32_t* perm_row, int T, int k, int vec_per_row,
+                                int sm_count, cudaStream_t st) {
+    const int blocks = min(ceil_div(T, 8), sm_count * 8);
+    if (blocks <= 0) return;
+    if (vec_per_row <= 32 * 8) scatter_rows_reg_kernel<8><<<blocks, 256, 0, st>>>(src, dst, perm_row, T, k, vec_per_row);
+    else if (vec_per_row <= 32 * 16) scatter_rows_reg_kernel<16><<<blocks, 256, 0, st>>>(src, dst, perm_row, T, k, vec_per_row);
+    else if (vec_per_row <= 32 * 28) scatter_rows_reg_kernel<28><<<blocks, 256, 0, st>>>(src, dst, perm_row, T, k, vec_per_row);
+    else if (vec_per_row <= 32 * 32) scatter_rows_reg_kernel<32><<<blocks, 256, 0, st>>>(src, dst, perm_row, T, k, vec_per_row);
+    else scatter_rows_kernel<<<blocks, 256, 0, st>>>(src, dst, perm_row, T, k, vec_per_row);
+}
+inline void launch_combine_rows(const uint4* Yp, const int32_t* perm_row, uint4* Y, int T, int k, int vec_per_row,
+                                int sm_count, cudaStream_t st) {
+    const int blocks = min(ceil_div(T, 8), sm_count * 8);
+    if (blocks <= 0) return;
+    // short rows (d < 4096) keep the chunked kernel: measured faster there (more warps per SM)
+    if (vec_per_row >= 32 * 16 && vec_per_row % (32 * 7) == 0)
+        combine_rows_seg_kernel<7><<<blocks, 256, 0, st>>>(Yp, perm_row, Y, T, k, vec_per_row);
+    else if (vec_per_row >= 32 * 16) combine_rows_seg_kernel<8><<<blocks, 256, 0, st>>>(Yp, perm_row, Y, T, k, vec_per_row);
+    else combine_rows_kernel<<<blocks, 256, 0, st>>>(Yp, perm_row, Y, T, k, vec_per_row);
+}
+
 // dgate[a] = sum over n-tiles of the partial dot products written by the dgrad-down epilogue
 // (row p = perm_row[a]; fixed order, so the result is reproducible).
 __global__ void dgate_reduce_kernel(const float* __restrict__ part, const int32_t* __restrict__ perm_row,
