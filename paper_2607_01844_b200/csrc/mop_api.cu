@@ -611,13 +611,17 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
                                                                                             s.E));
         if ((r = after_launch(c)) != MOP_OK) return r;
     }
+    if (units == 0) {   // nothing to permute: counts and offsets are all zero
+        LAUNCH(c, "perm_scan", st,
+               perm_scan_kernel<<<1, 1024, (s.E + 1) * sizeof(int32_t), st>>>(c->partial, counts, offsets, units, s.E));
+        return after_launch(c);
+    }
     LAUNCH(c, "perm_scan", st,
-           perm_scan_kernel<<<1, 1024, (s.E + 1) * sizeof(int32_t), st>>>(c->partial, counts, offsets, units, s.E));
+           perm_scan_cols_kernel<<<ceil_div(s.E, 32), PSCAN_WARPS * 32, 0, st>>>(c->partial, counts, units, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
-    if (units == 0) return MOP_OK;
     LAUNCH(c, "perm_rank", st,
-           perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, perm_row,
-                                                                                        row_src, M, s.E));
+           perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem + (s.E + 1) * sizeof(int32_t), st>>>(
+               topk_idx, c->partial, counts, offsets, perm_row, row_src, M, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
     if (!Xp) return MOP_OK;
     LAUNCH(c, "permute_scatter_rows", st,
@@ -1344,11 +1348,14 @@ mop_status mop_moe_permute_static(int device, int32_t T, int32_t d, int32_t E, i
         perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, M, E);
         if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
     }
-    perm_scan_kernel<<<1, 1024, (E + 1) * sizeof(int32_t), st>>>(su.scratch, counts, offsets, units, E);
+    if (units == 0) {
+        perm_scan_kernel<<<1, 1024, (E + 1) * sizeof(int32_t), st>>>(su.scratch, counts, offsets, units, E);
+        return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+    }
+    perm_scan_cols_kernel<<<ceil_div(E, 32), PSCAN_WARPS * 32, 0, st>>>(su.scratch, counts, units, E);
     if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
-    if (units == 0) return MOP_OK;
-    perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, su.scratch, perm_row, row_src,
-                                                                                M, E);
+    perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem + (E + 1) * sizeof(int32_t), st>>>(
+        topk_idx, su.scratch, counts, offsets, perm_row, row_src, M, E);
     if (cudaGetLastError() != cudaSuccess) return MOP_ERR_CUDA;
     if (!Xp) return MOP_OK;
     launch_scatter_rows(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, T, k, d / 8, su.sm_count, st);

@@ -31,8 +31,9 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_hist_kernel(const int32_
     for (int e = lane; e < E; e += 32) partial[(size_t)unit * E + e] = cnt[e];
 }
 
-// Scan: counts, offsets (exclusive scan over experts) and, in place of partial[u][e], the first
-// row of unit u inside expert e.  One block; thread e owns expert e (strided if E > blockDim).
+// Scan on one block: counts, offsets (exclusive scan over experts) and, in place of partial[u][e], the first
+// row of unit u inside expert e; thread e owns expert e (strided if E > blockDim).  Used when there is nothing
+// to permute (it still writes counts and offsets); otherwise perm_scan_cols_kernel + perm_rank_kernel do this.
 __global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ partial, int32_t* __restrict__ counts,
                                                          int32_t* __restrict__ offsets, int units, int E) {
     extern __shared__ int32_t scan_smem[];  // E + 1
@@ -72,18 +73,79 @@ __global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ p
     }
 }
 
-// Rank: second walk over the same segments; perm_row[a] = base[u][e] + rank inside the unit.
+// Column scan, spread over the GPU: a block owns 32 experts (a lane each: coalesced 128-byte rows of
+// partial[u][.]) and its eight warps own eight contiguous ranges of units.  In place of partial[u][e]: the
+// number of rows of expert e in the units before u; counts[e] = the expert's total.  Fixed order, no atomics.
+constexpr int PSCAN_WARPS = 8;
+__global__ void __launch_bounds__(PSCAN_WARPS * 32) perm_scan_cols_kernel(int32_t* __restrict__ partial,
+                                                                          int32_t* __restrict__ counts, int units,
+                                                                          int E) {
+    __shared__ int32_t tot[PSCAN_WARPS][32];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int e = blockIdx.x * 32 + lane;
+    const int per = (units + PSCAN_WARPS - 1) / PSCAN_WARPS;
+    const int u0 = min(units, warp * per), u1 = min(units, u0 + per);
+    int32_t run = 0;
+    if (e < E)
+        for (int u = u0; u < u1; ++u) {
+            const int32_t c = partial[(size_t)u * E + e];
+            partial[(size_t)u * E + e] = run;
+            run += c;
+        }
+    tot[warp][lane] = run;
+    __syncthreads();
+    int32_t before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < PSCAN_WARPS; ++w) {
+        if (w < warp) before += tot[w][lane];
+        total += tot[w][lane];
+    }
+    if (e < E) {
+        if (before)
+            for (int u = u0; u < u1; ++u) partial[(size_t)u * E + e] += before;
+        if (warp == 0) counts[e] = total;
+    }
+}
+
+// Rank: second walk over the same segments; perm_row[a] = offsets[e] + base[u][e] + rank inside the unit.
+// Every block scans counts[] into the experts' offsets for itself (E <= 1024 words of shared memory);
+// block 0 also writes them out.
 __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_t* __restrict__ idx,
                                                                     const int32_t* __restrict__ base,
+                                                                    const int32_t* __restrict__ counts,
+                                                                    int32_t* __restrict__ offsets,
                                                                     int32_t* __restrict__ perm_row,
                                                                     int32_t* __restrict__ row_src, int M, int E) {
     extern __shared__ int32_t perm_smem[];
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    int32_t* off = perm_smem + (size_t)PERM_WARPS * E;   // E + 1 words
+    for (int e = threadIdx.x; e < E; e += blockDim.x) off[e] = counts[e];
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive scan over E by one warp, 32 experts per step
+        int32_t carry = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane;
+            const int32_t c = (e < E) ? off[e] : 0;
+            int32_t inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += v;
+            }
+            if (e < E) off[e] = carry + inc - c;
+            carry += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) off[E] = carry;
+    }
+    __syncthreads();
+    if (blockIdx.x == 0)
+        for (int e = threadIdx.x; e <= E; e += blockDim.x) offsets[e] = off[e];
     int32_t* run = perm_smem + (size_t)warp * E;
     const int unit = blockIdx.x * PERM_WARPS + warp;
     const int a0 = unit * PERM_SEG;
     if (a0 >= M) return;
-    for (int e = lane; e < E; e += 32) run[e] = base[(size_t)unit * E + e];
+    for (int e = lane; e < E; e += 32) run[e] = base[(size_t)unit * E + e] + off[e];
     __syncwarp();
     const uint32_t lt = (1u << lane) - 1u;
     for (int it = 0; it < PERM_SEG / 32; ++it) {
