@@ -122,8 +122,10 @@ inline mop_status tc_ffn_bwd(TcPlan* p, const TcBwdArgs& a, int32_t* tiles, int3
         return MOP_OK;
     }
     mop_status r;
-    if ((r = tc_build_row_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
-    ++*launches;
+    if ((p->fwd_tn & 12) != 12) {   // row tiles of the tokens-on-M data gradients (the weight gradients need none)
+        if ((r = tc_build_row_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
+        ++*launches;
+    }
     CUtensorMap mWdKp, mWgKp, mWuKp;   // K-major weight maps boxed for a pair CTA (128 N rows)
     if (!tc_map_3d(p, &mWdKp, a.W_down, s.E, s.f, s.d, 128) || !tc_map_3d(p, &mWgKp, a.W_gate, s.E, s.d, s.f, 128) ||
         !tc_map_3d(p, &mWuKp, a.W_up, s.E, s.d, s.f, 128))

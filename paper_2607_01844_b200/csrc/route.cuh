@@ -385,7 +385,7 @@ constexpr int SELF_WARPS = 2;     // warps per block of the fast selection (a wa
 constexpr float ROUTE_EPS_C = 24.0f;      // order:  |z~ - z| <= C 2^-24 ||x_t|| max_e ||W_r[:,e]||  (see below)
 constexpr float ROUTE_EPS_GATE_C = 6.0f;  // gates:  the same with the largest error seen, not a bound (a tolerance, not an order)
 constexpr float ROUTE_GATE_REL = 5e-6f;   // a pick whose gate could be off by more than this (relative) gets its chain
-constexpr int SELF_XCHUNK = 256;  // elements of the token's row staged per step of the exact chains
+constexpr int SELF_XCHUNK = 512;  // elements of the token's row staged per step of the exact chains
 constexpr int SELF_CAND = 4;      // chains evaluated side by side (one lane each), their W_r^T rows staged in shared memory
 constexpr int SELF_WPITCH = SELF_XCHUNK + 4;   // row pitch of the staged W_r^T chunks: lanes read different banks
 constexpr int SELF_SMEM_FLOATS = SELF_XCHUNK + SELF_CAND * SELF_WPITCH;   // per warp, besides the 2 E logit / list words
@@ -551,11 +551,15 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t*
             // of W_r^T (lane l: 16-byte pieces l, l + 32, ... of the nc rows laid end to end).  The fetch of chunk
             // i + 1 is in flight while the chains run over chunk i.
             constexpr int WV = SELF_CAND * SELF_XCHUNK / 4 / 32;      // 16-byte pieces of W per lane and chunk
-            uint4 xq = make_uint4(0, 0, 0, 0);
+            constexpr int XV = SELF_XCHUNK / 8 / 32;                  // 16-byte pieces of x per lane and chunk
+            uint4 xq[XV];
             float4 wq[WV];
             auto fetch = [&](int i0) {
                 const int n = min(SELF_XCHUNK, d - i0);              // a multiple of 8
-                if (lane < n / 8) xq = __ldg(reinterpret_cast<const uint4*>(x + (size_t)t * d + i0) + lane);
+#pragma unroll
+                for (int u = 0; u < XV; ++u)
+                    if (lane + 32 * u < n / 8)
+                        xq[u] = __ldg(reinterpret_cast<const uint4*>(x + (size_t)t * d + i0) + lane + 32 * u);
 #pragma unroll
                 for (int u = 0; u < WV; ++u) {
                     const int v = lane + 32 * u, c = v / (SELF_XCHUNK / 4), j = v % (SELF_XCHUNK / 4);
@@ -567,10 +571,11 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t*
             for (int i0 = 0; i0 < d; i0 += SELF_XCHUNK) {
                 const int n = min(SELF_XCHUNK, d - i0);
                 __syncwarp();
-                {
-                    float* o = xs + lane * 8;
-                    o[0] = bf16_lo(xq.x); o[1] = bf16_hi(xq.x); o[2] = bf16_lo(xq.y); o[3] = bf16_hi(xq.y);
-                    o[4] = bf16_lo(xq.z); o[5] = bf16_hi(xq.z); o[6] = bf16_lo(xq.w); o[7] = bf16_hi(xq.w);
+#pragma unroll
+                for (int u = 0; u < XV; ++u) {
+                    float4* o = reinterpret_cast<float4*>(xs + (lane + 32 * u) * 8);
+                    o[0] = make_float4(bf16_lo(xq[u].x), bf16_hi(xq[u].x), bf16_lo(xq[u].y), bf16_hi(xq[u].y));
+                    o[1] = make_float4(bf16_lo(xq[u].z), bf16_hi(xq[u].z), bf16_lo(xq[u].w), bf16_hi(xq[u].w));
                 }
 #pragma unroll
                 for (int u = 0; u < WV; ++u) {
@@ -582,7 +587,7 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t*
                 if (mine) {
                     // the contract's chain: one fused multiply-add per i, i ascending
                     const float* wrow = ws + lane * SELF_WPITCH;
-#pragma unroll 4
+#pragma unroll 8
                     for (int i = 0; i < n; i += 4) {
                         const float4 w = *reinterpret_cast<const float4*>(wrow + i);
                         const float4 xv = *reinterpret_cast<const float4*>(xs + i);
