@@ -175,6 +175,42 @@ def test_all_keys_equal_goes_to_lowest_ids_and_leaves_experts_empty():
     check_integers(w, host, buf)
 
 
+def test_an_overflowing_expert_does_not_reach_its_neighbours_gradients():
+    """Backward with non-finite upstream gradients for the tokens of ONE expert (k = 1, so a token has one
+    expert): that expert's gradients are lost, every other expert's dW and every other token's dX and dgate
+    keep the bits of the clean run.  The rows of an expert end inside a 16-row K group of the weight-gradient
+    GEMMs for all but a few experts here, so the K tail of the expert before the poisoned one is exercised."""
+    w = synth.small("c5_train", T=1500, d=128, E=7, k=1, f=192, backward=True, seed=41)
+    host = synth.make_inputs(w, "cpu")
+    inp = to_dev(host)
+    for path in (binding.GEMM_AUTO, binding.GEMM_TENSOR_1CTA):
+        ctx = binding.context_for(w, gemm_path=path)
+        clean, bad = binding.LayerBuffers(w), binding.LayerBuffers(w)
+        binding.forward(ctx, inp, clean)
+        binding.backward(ctx, inp, clean)
+        counts = clean.counts.cpu().numpy()
+        e0 = int(np.argsort(counts)[len(counts) // 2])                    # an expert with rows, not the first one
+        if e0 == 0:
+            e0 = 1
+        assert counts[e0] > 0 and counts[e0 - 1] % 16 != 0
+        poisoned = dict(inp)
+        dY = inp["dY"].clone()
+        mine = (clean.idx[:, 0] == e0)
+        dY[mine] = float("inf")
+        dY[mine.nonzero()[::2, 0]] = float("nan")
+        poisoned["dY"] = dY
+        binding.forward(ctx, poisoned, bad)
+        binding.backward(ctx, poisoned, bad)
+        binding.mop_poll(ctx)
+        others = torch.ones(w.E, dtype=torch.bool, device="cuda")
+        others[e0] = False
+        for name in ("dW_gate", "dW_up", "dW_down"):
+            a, b = getattr(clean, name), getattr(bad, name)
+            assert torch.equal(a[others], b[others]), f"{name} of the other experts (path {path})"
+            assert not torch.isfinite(b[e0]).all(), f"{name} of the poisoned expert should be lost"
+        assert torch.equal(clean.dX[~mine], bad.dX[~mine]) and torch.equal(clean.dgate[~mine], bad.dgate[~mine])
+
+
 def test_zero_tokens_is_a_no_op():
     w = synth.small("c1_tiny", T=0, d=64, E=4, k=2, f=64, backward=True)
     host, inp, ctx, buf = run(w)
