@@ -43,6 +43,7 @@ struct mop_ctx {
     bf16* fr_pieces;
     float *fr_wrT, *fr_colsq, *fr_xnorm, *fr_scal, *fr_wsq;
     int32_t* fr_todo;
+    int fr_rblocks;          // resident blocks of the resolving pass
     // host-buffer entry point scratch
     bf16 *hx, *hXp, *hH, *hYp, *hY, *hG, *hU, *hdY, *hdX;
     int32_t *hidx, *hcounts, *hoffsets, *hperm, *hsrc;
@@ -403,6 +404,7 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         if (st != MOP_OK) { cudaFree(c->ws); delete c; return st; }
         if (c->fast_route) {
             bool ok = cudaMemset(c->fr_scal, 0, 256) == cudaSuccess;
+            c->fr_rblocks = route_resolve_resident(shape->E, c->sm_count);
             ok = ok && cudaStreamCreateWithFlags(&c->fr_stream, cudaStreamNonBlocking) == cudaSuccess &&
                  cudaEventCreateWithFlags(&c->fr_fork, cudaEventDisableTiming) == cudaSuccess &&
                  cudaEventCreateWithFlags(&c->fr_join, cudaEventDisableTiming) == cudaSuccess;
@@ -553,7 +555,7 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
         int32_t* stats = reinterpret_cast<int32_t*>(c->fr_scal) + 8;
         int32_t* n_todo = reinterpret_cast<int32_t*>(c->fr_scal) + 16;
         CUDA_OK(cudaMemsetAsync(n_todo, 0, 4, st));
-        const int rblocks = min(ceil_div(s.T, SELF_WARPS), c->sm_count * 12);
+        const int rblocks = min(ceil_div(s.T, SELF_WARPS), c->fr_rblocks);
         LAUNCH(c, "route_select_screen", st,
                route_select_fast(z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
                                  c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 0, rblocks, st));

@@ -712,6 +712,25 @@ inline void route_select_fast_q(float* z, const float* bias, const bf16* x, cons
                                                                                 n_todo, stats, d, E, k, score_fn, bias_mode);
     }
 }
+// Blocks of the resolving pass that are resident at once: its grid.  Every warp then walks its share of the list;
+// a larger grid would run in waves of whole walks.
+template <int Q>
+inline int route_resolve_resident_q(int E, int sm_count) {
+    int nb = 0;
+    const size_t smem = (size_t)SELF_WARPS * (2 * E + SELF_SMEM_FLOATS) * sizeof(float);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, route_resolve_kernel<Q>, SELF_WARPS * 32, smem) != cudaSuccess || nb < 1)
+        nb = 1;
+    return nb * sm_count;
+}
+inline int route_resolve_resident(int E, int sm_count) {
+    const int q = ceil_div(E, 32);
+    if (q <= 2) return route_resolve_resident_q<2>(E, sm_count);
+    if (q <= 4) return route_resolve_resident_q<4>(E, sm_count);
+    if (q <= 8) return route_resolve_resident_q<8>(E, sm_count);
+    if (q <= 12) return route_resolve_resident_q<12>(E, sm_count);
+    if (q <= 16) return route_resolve_resident_q<16>(E, sm_count);
+    return route_resolve_resident_q<32>(E, sm_count);
+}
 inline void route_select_fast(float* z, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
                               const float* wsq, int32_t* idx, float* gate, int32_t* todo, int32_t* n_todo, int32_t* stats,
                               int T, int d, int E, int k, int score_fn, int bias_mode, int pass, int resolve_blocks,
