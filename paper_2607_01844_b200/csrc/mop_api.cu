@@ -540,15 +540,17 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
         // re-evaluated where the order is in doubt
         mop_status r;
         dim3 gp(ceil_div(s.E, 32), ceil_div(s.d, 32));
-        // the row norms of x depend on nothing else: they run on a side stream beside the logit GEMM
+        LAUNCH(c, "route_prep", st,
+               route_prep_kernel<<<gp, 256, 0, st>>>(W_r, c->fr_pieces, c->fr_wrT, c->fr_colsq, s.d, s.E));
+        if ((r = after_launch(c)) != MOP_OK) return r;
+        // only the selection needs the norms of x's rows and of W_r's columns: they run on a side stream beside
+        // the logit GEMM (which leaves room on every SM for such blocks, and DRAM idle)
         CUDA_OK(cudaEventRecord(c->fr_fork, st));
         CUDA_OK(cudaStreamWaitEvent(c->fr_stream, c->fr_fork, 0));
+        route_wnorm_kernel<<<ceil_div(s.E, 8), 256, 0, c->fr_stream>>>(c->fr_colsq, c->fr_wsq, ceil_div(s.d, 32), s.E);
         route_xnorm_kernel<<<ceil_div(s.T, 8), 256, 0, c->fr_stream>>>(static_cast<const bf16*>(x), c->fr_xnorm, s.T, s.d);
         CUDA_OK(cudaEventRecord(c->fr_join, c->fr_stream));
-        LAUNCH(c, "route_prep", st,
-               route_prep_kernel<<<gp, 256, 0, st>>>(W_r, c->fr_pieces, c->fr_wrT, c->fr_colsq, s.d, s.E);
-               route_wnorm_kernel<<<ceil_div(s.E, 8), 256, 0, st>>>(c->fr_colsq, c->fr_wsq, ceil_div(s.d, 32), s.E));
-        if ((r = after_launch(c, 3)) != MOP_OK) return r;
+        c->launches += 2;
         if ((r = rs_launch(&c->plan, "route_score_tc", x, c->fr_pieces, z, s.T, s.d, s.E, c->status, st)) != MOP_OK) return r;
         c->launches += 1;
         CUDA_OK(cudaStreamWaitEvent(st, c->fr_join, 0));
