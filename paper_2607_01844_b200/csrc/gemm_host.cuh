@@ -63,13 +63,19 @@ inline mop_status tc_ffn_fwd_impl(TcPlan* p, const TcFwdArgs& a, int32_t* tiles,
     // Tokens-on-N kernels: fwd_tn bit 0 = up-projection, bit 1 = down-projection (see tc_plan_policy)
     const bool gather = a.x_gather != nullptr;
     const bool tn_f1 = gather || (p->fwd_tn & 1), tn_f2 = p->fwd_tn & 2;
-    if (tn_f1 || tn_f2) {
-        if ((r = tn_build_tiles(p, a.offsets, tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4), st)) != MOP_OK) return r;
+    int32_t* ttiles_fwd = tiles + 2 * (tc_tile_table_bytes(s.T * s.k, s.E) / 4);
+    if ((tn_f1 != tn_f2) && p->pairs == 0) {   // one GEMM on each kind of kernel: both tables in one launch
+        if ((r = build_both_tiles(p, a.offsets, tiles, ttiles_fwd, st)) != MOP_OK) return r;
         ++*launches;
-    }
-    if (!tn_f1 || !tn_f2) {
-        if ((r = tc_build_row_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
-        ++*launches;
+    } else {
+        if (tn_f1 || tn_f2) {
+            if ((r = tn_build_tiles(p, a.offsets, ttiles_fwd, st)) != MOP_OK) return r;
+            ++*launches;
+        }
+        if (!tn_f1 || !tn_f2) {
+            if ((r = tc_build_row_tiles(p, a.offsets, tiles, st)) != MOP_OK) return r;
+            ++*launches;
+        }
     }
     // N-major weights as chunked maps: one-CTA tiles take 2 chunks per tensor (gate | up) or 4 (down);
     // a pair CTA takes 2 chunks

@@ -354,10 +354,9 @@ __device__ __forceinline__ TileInfo decode_tile(const TcArgs& a, int t) {
 }
 
 // 128-row tile list of the ragged-M GEMMs, built on the device from offsets (no host round trip).
-__global__ void __launch_bounds__(1024) tc_build_mtiles_kernel(const int32_t* __restrict__ offsets, int E,
-                                                               int4* __restrict__ mtiles,
-                                                               int32_t* __restrict__ n_mtiles) {
-    __shared__ int32_t scan[1025];
+__device__ __forceinline__ void tc_build_mtiles_body(const int32_t* __restrict__ offsets, int E,
+                                                     int4* __restrict__ mtiles, int32_t* __restrict__ n_mtiles,
+                                                     int32_t* scan) {
     const int e = threadIdx.x;
     int cnt = 0, off = 0;
     if (e < E) { off = offsets[e]; cnt = offsets[e + 1] - off; }
@@ -374,6 +373,12 @@ __global__ void __launch_bounds__(1024) tc_build_mtiles_kernel(const int32_t* __
     const int first = scan[e] - nt;
     for (int i = 0; i < nt; ++i) mtiles[first + i] = make_int4(e, off + i * TC_BM, min(TC_BM, cnt - i * TC_BM), 0);
     if (e == 1023) *n_mtiles = scan[1023];
+}
+__global__ void __launch_bounds__(1024) tc_build_mtiles_kernel(const int32_t* __restrict__ offsets, int E,
+                                                               int4* __restrict__ mtiles,
+                                                               int32_t* __restrict__ n_mtiles) {
+    __shared__ int32_t scan[1025];
+    tc_build_mtiles_body(offsets, E, mtiles, n_mtiles, scan);
 }
 
 // Epilogue of one 128 x 256 accumulator for the kinds whose rows are token rows: this thread owns

@@ -56,10 +56,9 @@ struct TnArgs {
 };
 
 // Token tiles: an expert's rows are cut into ceil(rows/256) nearly equal tiles.
-__global__ void __launch_bounds__(1024) tn_build_ttiles_kernel(const int32_t* __restrict__ offsets, int E,
-                                                               int4* __restrict__ tiles,
-                                                               int32_t* __restrict__ n_tiles) {
-    __shared__ int32_t scan[1024];
+__device__ __forceinline__ void tn_build_ttiles_body(const int32_t* __restrict__ offsets, int E,
+                                                     int4* __restrict__ tiles, int32_t* __restrict__ n_tiles,
+                                                     int32_t* scan) {
     const int e = threadIdx.x;
     int cnt = 0, off = 0;
     if (e < E) { off = offsets[e]; cnt = offsets[e + 1] - off; }
@@ -77,6 +76,20 @@ __global__ void __launch_bounds__(1024) tn_build_ttiles_kernel(const int32_t* __
     // .w = position of the tile within its expert | number of tiles of the expert << 16
     for (int i = 0; i < nt; ++i) tiles[first + i] = make_int4(e, off + i * sz, min(sz, cnt - i * sz), i | (nt << 16));
     if (e == 1023) *n_tiles = scan[1023];
+}
+__global__ void __launch_bounds__(1024) tn_build_ttiles_kernel(const int32_t* __restrict__ offsets, int E,
+                                                               int4* __restrict__ tiles,
+                                                               int32_t* __restrict__ n_tiles) {
+    __shared__ int32_t scan[1025];
+    tn_build_ttiles_body(offsets, E, tiles, n_tiles, scan);
+}
+// Both tables in one launch (block 0: 128-row tiles of the tokens-on-M kernels, block 1: token tiles).
+__global__ void __launch_bounds__(1024) build_both_tiles_kernel(const int32_t* __restrict__ offsets, int E,
+                                                                int4* __restrict__ mtiles, int32_t* __restrict__ n_mtiles,
+                                                                int4* __restrict__ ttiles, int32_t* __restrict__ n_ttiles) {
+    __shared__ int32_t scan[1025];
+    if (blockIdx.x == 0) tc_build_mtiles_body(offsets, E, mtiles, n_mtiles, scan);
+    else tn_build_ttiles_body(offsets, E, ttiles, n_ttiles, scan);
 }
 
 // Four rows of a [rows, cols] bf16 tensor (map box {64, 1}) -> 4 x 128 bytes at dst, swizzled like a tile box.
@@ -490,6 +503,13 @@ inline mop_status tn_init() {
     return MOP_OK;
 }
 
+inline mop_status build_both_tiles(TcPlan* p, const int32_t* offsets, int32_t* mtiles, int32_t* ttiles, cudaStream_t st) {
+    p->prof->begin("build_tiles", st);
+    build_both_tiles_kernel<<<2, 1024, 0, st>>>(offsets, p->s.E, reinterpret_cast<int4*>(mtiles + 64), mtiles,
+                                                reinterpret_cast<int4*>(ttiles + 64), ttiles);
+    p->prof->end(st);
+    return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
+}
 inline mop_status tn_build_tiles(TcPlan* p, const int32_t* offsets, int32_t* tiles, cudaStream_t st) {
     p->prof->begin("tn_build_ttiles", st);
     tn_build_ttiles_kernel<<<1, 1024, 0, st>>>(offsets, p->s.E, reinterpret_cast<int4*>(tiles + 64), tiles);

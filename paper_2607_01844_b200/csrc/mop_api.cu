@@ -609,6 +609,12 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
     const int units = perm_units(s);
     const size_t smem = (size_t)PERM_WARPS * s.E * sizeof(int32_t);
     mop_status r;
+    if (perm_small_fits(units, s.E)) {   // a few units: one block does histogram, scan and rank
+        LAUNCH(c, "perm_small", st,
+               perm_small_kernel<<<1, 1024, ((size_t)units * s.E + s.E + 1) * sizeof(int32_t), st>>>(
+                   topk_idx, counts, offsets, perm_row, row_src, M, s.E, units));
+        if ((r = after_launch(c)) != MOP_OK) return r;
+    } else {
     if (units > 0) {
         LAUNCH(c, "perm_hist", st,
                perm_hist_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem, st>>>(topk_idx, c->partial, M,
@@ -627,6 +633,7 @@ mop_status mop_moe_permute(mop_ctx* c, const void* x, const int32_t* topk_idx, i
            perm_rank_kernel<<<ceil_div(units, PERM_WARPS), PERM_WARPS * 32, smem + (s.E + 1) * sizeof(int32_t), st>>>(
                topk_idx, c->partial, counts, offsets, perm_row, row_src, M, s.E));
     if ((r = after_launch(c)) != MOP_OK) return r;
+    }
     if (!Xp) return MOP_OK;
     LAUNCH(c, "permute_scatter_rows", st,
            launch_scatter_rows(static_cast<const uint4*>(x), static_cast<uint4*>(Xp), perm_row, s.T, s.k, s.d / 8,

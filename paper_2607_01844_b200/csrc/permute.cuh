@@ -165,6 +165,87 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_
     }
 }
 
+// Small layers: histogram, scan and rank in ONE block (the three launches above cost more than their work when
+// there are only a few units).  Warp w owns the units w, w + 32, ...; cnt[u][e] lives in shared memory, first as
+// the unit's histogram, then as the first row of unit u inside expert e.  Same tables as the three-kernel path.
+constexpr int PERM_SMALL_MAX_UNITS = 8;       // beyond that the three parallel kernels are faster (measured at 48 units)
+constexpr int PERM_SMALL_MAX_WORDS = 10240;     // units * E words of shared memory (40 KiB)
+__global__ void __launch_bounds__(1024) perm_small_kernel(const int32_t* __restrict__ idx, int32_t* __restrict__ counts,
+                                                          int32_t* __restrict__ offsets, int32_t* __restrict__ perm_row,
+                                                          int32_t* __restrict__ row_src, int M, int E, int units) {
+    extern __shared__ int32_t perm_smem[];
+    int32_t* cnt = perm_smem;                      // [units][E]
+    int32_t* off = perm_smem + (size_t)units * E;  // [E + 1]
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    for (int i = threadIdx.x; i < units * E; i += blockDim.x) cnt[i] = 0;
+    __syncthreads();
+    for (int u = warp; u < units; u += 32) {
+        int32_t* c = cnt + (size_t)u * E;
+        for (int it = 0; it < PERM_SEG / 32; ++it) {
+            const int a = u * PERM_SEG + it * 32 + lane;
+            int e = (a < M) ? idx[a] : -1;
+            if (e < 0 || e >= E) e = -1;
+            const uint32_t same = __match_any_sync(0xffffffffu, e);
+            if (e >= 0 && lane == __ffs(same) - 1) c[e] += __popc(same);
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        int32_t run = 0;
+        for (int u = 0; u < units; ++u) {
+            const int32_t c = cnt[(size_t)u * E + e];
+            cnt[(size_t)u * E + e] = run;
+            run += c;
+        }
+        counts[e] = run;
+        off[e] = run;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int32_t carry = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + lane;
+            const int32_t c = (e < E) ? off[e] : 0;
+            int32_t inc = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += v;
+            }
+            if (e < E) off[e] = carry + inc - c;
+            carry += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) off[E] = carry;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) offsets[e] = off[e];
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int u = warp; u < units; u += 32) {
+        int32_t* run = cnt + (size_t)u * E;
+        for (int e = lane; e < E; e += 32) run[e] += off[e];
+        __syncwarp();
+        for (int it = 0; it < PERM_SEG / 32; ++it) {
+            const int a = u * PERM_SEG + it * 32 + lane;
+            int e = (a < M) ? idx[a] : -1;
+            if (e < 0 || e >= E) e = -1;
+            const uint32_t same = __match_any_sync(0xffffffffu, e);
+            int32_t p = -1;
+            if (e >= 0) p = run[e] + __popc(same & lt);
+            __syncwarp();
+            if (e >= 0 && lane == __ffs(same) - 1) run[e] += __popc(same);
+            __syncwarp();
+            if (a < M) {
+                perm_row[a] = p;
+                if (p >= 0) row_src[p] = a;
+            }
+        }
+    }
+}
+inline bool perm_small_fits(int units, int E) {
+    return units > 0 && units <= PERM_SMALL_MAX_UNITS && (long long)units * E <= PERM_SMALL_MAX_WORDS;
+}
+
 // Scatter rows: one warp per token reads x[t,:] once (16-byte vectors, coalesced) and writes it to
 // its k destination rows.  Used for x -> Xp and for dY -> dYp.
 __global__ void __launch_bounds__(256) scatter_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
