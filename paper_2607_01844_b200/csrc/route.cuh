@@ -571,12 +571,11 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t*
             for (int i0 = 0; i0 < d; i0 += SELF_XCHUNK) {
                 const int n = min(SELF_XCHUNK, d - i0);
                 __syncwarp();
+                // x stays bf16 in shared memory (16 bytes = 8 elements per load in the chains: every shared-memory
+                // instruction of a warp costs a wavefront however few lanes take part, and the chains of all
+                // resident warps together are bound by those wavefronts when most tokens are listed)
 #pragma unroll
-                for (int u = 0; u < XV; ++u) {
-                    float4* o = reinterpret_cast<float4*>(xs + (lane + 32 * u) * 8);
-                    o[0] = make_float4(bf16_lo(xq[u].x), bf16_hi(xq[u].x), bf16_lo(xq[u].y), bf16_hi(xq[u].y));
-                    o[1] = make_float4(bf16_lo(xq[u].z), bf16_hi(xq[u].z), bf16_lo(xq[u].w), bf16_hi(xq[u].w));
-                }
+                for (int u = 0; u < XV; ++u) reinterpret_cast<uint4*>(xs)[lane + 32 * u] = xq[u];
 #pragma unroll
                 for (int u = 0; u < WV; ++u) {
                     const int v = lane + 32 * u, c = v / (SELF_XCHUNK / 4), j = v % (SELF_XCHUNK / 4);
@@ -587,14 +586,19 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t*
                 if (mine) {
                     // the contract's chain: one fused multiply-add per i, i ascending
                     const float* wrow = ws + lane * SELF_WPITCH;
-#pragma unroll 8
-                    for (int i = 0; i < n; i += 4) {
-                        const float4 w = *reinterpret_cast<const float4*>(wrow + i);
-                        const float4 xv = *reinterpret_cast<const float4*>(xs + i);
-                        acc = __fmaf_rn(xv.x, w.x, acc);
-                        acc = __fmaf_rn(xv.y, w.y, acc);
-                        acc = __fmaf_rn(xv.z, w.z, acc);
-                        acc = __fmaf_rn(xv.w, w.w, acc);
+#pragma unroll 4
+                    for (int i = 0; i < n; i += 8) {
+                        const float4 w0 = *reinterpret_cast<const float4*>(wrow + i);
+                        const float4 w1 = *reinterpret_cast<const float4*>(wrow + i + 4);
+                        const uint4 xv = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(xs) + i);
+                        acc = __fmaf_rn(bf16_lo(xv.x), w0.x, acc);
+                        acc = __fmaf_rn(bf16_hi(xv.x), w0.y, acc);
+                        acc = __fmaf_rn(bf16_lo(xv.y), w0.z, acc);
+                        acc = __fmaf_rn(bf16_hi(xv.y), w0.w, acc);
+                        acc = __fmaf_rn(bf16_lo(xv.z), w1.x, acc);
+                        acc = __fmaf_rn(bf16_hi(xv.z), w1.y, acc);
+                        acc = __fmaf_rn(bf16_lo(xv.w), w1.z, acc);
+                        acc = __fmaf_rn(bf16_hi(xv.w), w1.w, acc);
                     }
                 }
             }
