@@ -14,7 +14,7 @@ def pytest_configure(config):
 
 
 def pytest_terminal_summary(terminalreporter):
-    """Realised float errors of the GPU parity checks: written to gpurun_out/parity_errors.json and summarised."""
+    """Realised float errors of the GPU parity checks: written to parity_errors.json in the output folder and summarised."""
     sys.path.insert(0, str(Path(__file__).resolve().parent))
     import parity_util
     table = parity_util.dump()

@@ -24,8 +24,8 @@ experts picked by row count):
          rows, |dW| up to 33) plus 1e-3 |ref|.
   dX_voc, dW_voc  the same two cases for the vocabulary projection (dX bf16: realised 0.031 at |ref| <= 10;
          dW_voc fp32: one flipped dY of size 1.5 times |x| = 3 is 0.02).
-Every check is recorded (tensor, case, realised errors) and written to gpurun_out/parity_errors.json
-when the session ends.
+Every check is recorded (tensor, case, realised errors) and written to parity_errors.json in the output
+folder when the session ends.
 """
 import json
 from pathlib import Path
