@@ -36,6 +36,8 @@ constexpr int RS_SMEM_BYTES = (RS_SA + RS_SB) * RS_SLOT + 1024 /*align*/ + TC_BA
 
 struct RsArgs {
     float* z;          // [T, E] fp32 logits (device)
+    float* z1;         // splits == 2: the sum over the second half of K goes here (the selection adds the two)
+    int splits;        // 1 or 2 halves of the K loop per tile, as separate units of work
     int T, d, E;
     int32_t* status;
 };
@@ -81,23 +83,45 @@ route_score_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
 
     const int kblocks = args.d / TC_BK;
-    const int tiles_n = (args.E + 255) / 256;
-    const int total_tiles = ((args.T + 255) / 256) * tiles_n;
+    const int tiles_n = (args.E + 255) / 256, tiles_m = (args.T + 255) / 256;
+    const int total_tiles = tiles_m * tiles_n * args.splits;
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
     // columns of n-tile nt: 256, or 128 for a last tile of at most 128 columns
     auto tile_cols = [&](int nt) { return (args.E - 256 * nt <= 128) ? 128 : 256; };
+    // Unit of work t -> block of tokens, n-tile, half of K.  The 256-column tiles come first and the narrow last
+    // ones after them (they cost half as much: the round-robin over the pairs then ends evenly); the halves of K of
+    // one tile are neighbours, and so are the tiles of one block of tokens: x is read from DRAM once.
+    const int wide_n = tiles_n - (tile_cols(tiles_n - 1) == 128 ? 1 : 0);
+    const int wide_units = tiles_m * wide_n * args.splits;
+    struct Unit { int mt, nt, kb0, kb1; float* out; };
+    auto decode = [&](int t) {
+        Unit u;
+        int r, nn, n_first;
+        if (t < wide_units) { r = t; nn = wide_n; n_first = 0; }
+        else { r = t - wide_units; nn = tiles_n - wide_n; n_first = wide_n; }
+        const int ks = r % args.splits;
+        r /= args.splits;
+        u.mt = r / nn;
+        u.nt = n_first + (r - u.mt * nn);
+        const int per = (kblocks + args.splits - 1) / args.splits;
+        u.kb0 = ks * per;
+        u.kb1 = min(kblocks, u.kb0 + per);
+        u.out = ks ? args.z1 : args.z;
+        return u;
+    };
 
     if (warp == 0) {
         // ===================================================================== TMA producer (both CTAs)
         if (lane == 0) {
             int sa = 0, sb = 0; uint32_t pa = 0, pb = 0; bool alive = true;
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
-                const int mt = t / tiles_n, nt = t - mt * tiles_n;
-                const int row0 = mt * 256 + 128 * (int)rank;          // past T: the copy fills zeros
+                const Unit u = decode(t);
+                const int nt = u.nt;
+                const int row0 = u.mt * 256 + 128 * (int)rank;        // past T: the copy fills zeros
                 const int half_cols = tile_cols(nt) >> 1;             // this CTA's columns: 64 or 128
                 const int chunk0 = (nt * 256 + (int)rank * half_cols) >> 6;
                 const CUtensorMap* mw = half_cols == 128 ? &tmW2 : &tmW1;
-                for (int kb = 0; kb < kblocks && alive; ++kb) {
+                for (int kb = u.kb0; kb < u.kb1 && alive; ++kb) {
                     if (!mbar_wait(emptyA(sa), pa ^ 1u, abort_flag, args.status, STATUS_WAIT_EMPTY)) { alive = false; break; }
                     if (leader) mbar_expect_tx(fullA(sa), 2 * RS_SLOT);
                     tma2_load_2d(slotA(sa), &tmX, fullA(sa) & T2_PEER_MASK, kb * TC_BK, row0);
@@ -122,14 +146,14 @@ route_score_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
             constexpr uint32_t b_step = 2048 >> 4;      // 16 rows of K, 128 bytes each
             int sa = 0, sb = 0; uint32_t pa = 0, pb = 0; int it = 0; bool alive = true;
             for (int t = cluster_id; t < total_tiles && alive; t += n_clusters) {
-                const int nt = t % tiles_n;
-                const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(nt) >> 3) << 17);
+                const Unit u = decode(t);
+                const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(u.nt) >> 3) << 17);
                 if (!mbar_wait(tempty_bar(it & 1), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag, args.status,
                                STATUS_WAIT_TMEM_EMPTY)) break;
                 tc_fence_after();
                 uint32_t d_tmem = tmem_base + (uint32_t)(it & 1) * TC_BN;
                 int kseg = 0;                            // K block inside the segment
-                for (int kb = 0; kb < kblocks && alive; ++kb) {
+                for (int kb = u.kb0; kb < u.kb1 && alive; ++kb) {
                     if (!mbar_wait(fullA(sa), pa, abort_flag, args.status, STATUS_WAIT_FULL)) { alive = false; break; }
                     const uint64_t da = desc_a | (uint64_t)((slotA(sa) & 0x3ffffu) >> 4);
                     for (int ph = 0; ph < 3; ++ph) {
@@ -145,7 +169,7 @@ route_score_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
                     if (!alive) break;
                     umma2_commit_both(emptyA(sa));
                     if (++sa == RS_SA) { sa = 0; pa ^= 1u; }
-                    if (++kseg == RS_SEG && kb + 1 < kblocks) {
+                    if (++kseg == RS_SEG && kb + 1 < u.kb1) {
                         // segment done: hand this accumulator to the epilogue and go on in the other one
                         umma2_commit_both(tfull_bar(it & 1));
                         ++it;
@@ -165,11 +189,12 @@ route_score_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
         // ===================================================================== epilogue (8 warps, both CTAs)
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 belong to this warp
         const int half = (warp - 2) >> 2;        // columns [128*half, 128*half + 128) of the tile
-        const int nseg = (kblocks + RS_SEG - 1) / RS_SEG;
         int it = 0;
         bool ok = true;
         for (int t = cluster_id; t < total_tiles && ok; t += n_clusters) {
-            const int mt = t / tiles_n, nt = t - mt * tiles_n;
+            const Unit u = decode(t);
+            const int mt = u.mt, nt = u.nt;
+            const int nseg = (u.kb1 - u.kb0 + RS_SEG - 1) / RS_SEG;
             const bool active = half * 128 < tile_cols(nt);
             float sum[4][32];
 #pragma unroll
@@ -202,7 +227,7 @@ route_score_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_co
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     const int col = nt * 256 + half * 128 + 32 * g;
-                    if (col < args.E) epi_f32<32>(args.z + (size_t)row * args.E + col, sum[g], 0);
+                    if (col < args.E) epi_f32<32>(u.out + (size_t)row * args.E + col, sum[g], 0);
                 }
             }
         }
@@ -228,16 +253,45 @@ inline mop_status rs_init() {
                    cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }
 
-// x: [T, d] bf16; pieces: [3, d, E] bf16; z: [T, E] fp32 (all device).  d and E multiples of 64.
-inline mop_status rs_launch(const TcPlan* p, const char* name, const void* x, const void* pieces, float* z, int T, int d,
-                            int E, int32_t* status, cudaStream_t st) {
+// Halves of K as separate units pay when the tiles leave many pairs idle or end unevenly (config 5: 32 wide and 32
+// narrow tiles on 74 pairs: the last pair finishes after 0.75 instead of 1 tile time); the makespan of the
+// kernel's round-robin is computed for both and the shorter one taken.
+inline int rs_pick_splits(int T, int d, int E, int n_clusters) {
+    const int tiles_m = (T + 255) / 256, tiles_n = (E + 255) / 256;
+    const bool narrow_last = E - 256 * (tiles_n - 1) <= 128;
+    const int wide_n = tiles_n - (narrow_last ? 1 : 0);
+    if (d / TC_BK < 2 * RS_SEG || n_clusters < 1) return 1;
+    double best = 0.0;
+    int pick = 1;
+    for (int splits = 1; splits <= 2; ++splits) {
+        const int wide = tiles_m * wide_n * splits, total = tiles_m * tiles_n * splits;
+        double worst = 0.0;
+        for (int c = 0; c < n_clusters && c < total; ++c) {
+            double sum = 0.0;
+            for (int t = c; t < total; t += n_clusters) sum += (t < wide ? 1.0 : 0.5) / splits;
+            worst = sum > worst ? sum : worst;
+        }
+        worst += 0.03 * (splits - 1);     // a second partial sum costs a little in the selection
+        if (splits == 1 || worst < 0.9 * best) { best = worst; pick = splits; }
+    }
+    return pick;
+}
+
+// x: [T, d] bf16; pieces: [3, d, E] bf16; z, z1: [T, E] fp32 (all device).  d and E multiples of 64.
+// Returns in *used_splits whether the logits are z (1) or z + z1 (2).
+inline mop_status rs_launch(const TcPlan* p, const char* name, const void* x, const void* pieces, float* z, float* z1,
+                            int T, int d, int E, int32_t* status, int* used_splits, cudaStream_t st) {
     CUtensorMap mX, mW2, mW1;
     if (!tc_map_2d(p, &mX, x, T, d, 128) || !tc_map_chunked_3d(p, &mW2, pieces, 3, d, E, 2) ||
         !tc_map_chunked_3d(p, &mW1, pieces, 3, d, E, 1))
         return MOP_ERR_CUDA;
-    RsArgs a{z, T, d, E, status};
+    const int grid = p->sm_count & ~1;
+    RsArgs a{};
+    a.z = z; a.z1 = z1; a.T = T; a.d = d; a.E = E; a.status = status;
+    a.splits = z1 ? rs_pick_splits(T, d, E, grid / 2) : 1;
+    *used_splits = a.splits;
     p->prof->begin(name, st);
-    route_score_pair_kernel<<<p->sm_count & ~1, RS_THREADS, RS_SMEM_BYTES, st>>>(mX, mW2, mW1, a);
+    route_score_pair_kernel<<<grid, RS_THREADS, RS_SMEM_BYTES, st>>>(mX, mW2, mW1, a);
     p->prof->end(st);
     return cudaGetLastError() == cudaSuccess ? MOP_OK : MOP_ERR_CUDA;
 }

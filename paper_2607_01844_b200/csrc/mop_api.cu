@@ -41,7 +41,7 @@ struct mop_ctx {
     cudaStream_t fr_stream;          // the row norms of x are taken beside the logit GEMM
     cudaEvent_t fr_fork, fr_join;
     bf16* fr_pieces;
-    float *fr_wrT, *fr_colsq, *fr_xnorm, *fr_scal, *fr_wsq;
+    float *fr_wrT, *fr_colsq, *fr_xnorm, *fr_scal, *fr_wsq, *fr_z1;
     int32_t* fr_todo;
     int fr_rblocks;          // resident blocks of the resolving pass
     // host-buffer entry point scratch
@@ -77,7 +77,7 @@ constexpr uint32_t GUARD_PATTERN = 0xA5C3A5C3u;
 
 struct Layout {
     size_t z, partial, tiles, status, part, dYp, dG, dU, gH, dXp, dz_sel, dz_row, wrT, rG, rU, rH;
-    size_t fr_pieces, fr_wrT, fr_colsq, fr_xnorm, fr_scal, fr_wsq, fr_todo;
+    size_t fr_pieces, fr_wrT, fr_colsq, fr_xnorm, fr_scal, fr_wsq, fr_todo, fr_z1;
     size_t hx, hXp, hH, hYp, hY, hidx, hcounts, hoffsets, hperm, hsrc, hgate;
     size_t hG, hU, hdY, hdX, hdgate;
     size_t qx, qY, qidx, qgate, qdY, qdX, qdgate;   // second slot of the pipelined host entry points
@@ -134,6 +134,7 @@ Layout make_layout(const mop_moe_shape& s) {
         L.fr_scal = take(256);
         L.fr_wsq = take(E * 4);
         L.fr_todo = take(T * 4 + 16);
+        L.fr_z1 = take(T * E * 4);
     }
     if (s.with_backward) {
         L.part = take((size_t)part_tiles(s) * M * 4);
@@ -319,6 +320,7 @@ mop_status mop_create(mop_ctx** out, const mop_moe_shape* shape, int device) {
         c->fr_scal = reinterpret_cast<float*>(w + L.fr_scal);
         c->fr_wsq = reinterpret_cast<float*>(w + L.fr_wsq);
         c->fr_todo = reinterpret_cast<int32_t*>(w + L.fr_todo);
+        c->fr_z1 = reinterpret_cast<float*>(w + L.fr_z1);
         c->fast_route = route_fast_wanted(*shape);
     } else if (shape->route_path == MOP_ROUTE_TENSOR) {
         cudaFree(c->ws); delete c;
@@ -551,7 +553,10 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
         route_xnorm_kernel<<<ceil_div(s.T, 8), 256, 0, c->fr_stream>>>(static_cast<const bf16*>(x), c->fr_xnorm, s.T, s.d);
         CUDA_OK(cudaEventRecord(c->fr_join, c->fr_stream));
         c->launches += 2;
-        if ((r = rs_launch(&c->plan, "route_score_tc", x, c->fr_pieces, z, s.T, s.d, s.E, c->status, st)) != MOP_OK) return r;
+        int splits = 1;
+        if ((r = rs_launch(&c->plan, "route_score_tc", x, c->fr_pieces, z, c->fr_z1, s.T, s.d, s.E, c->status, &splits, st)) != MOP_OK)
+            return r;
+        const float* z1 = splits == 2 ? c->fr_z1 : nullptr;
         c->launches += 1;
         CUDA_OK(cudaStreamWaitEvent(st, c->fr_join, 0));
         int32_t* stats = reinterpret_cast<int32_t*>(c->fr_scal) + 8;
@@ -559,12 +564,14 @@ mop_status mop_moe_route(mop_ctx* c, const void* x, const float* W_r, const floa
         CUDA_OK(cudaMemsetAsync(n_todo, 0, 4, st));
         const int rblocks = min(ceil_div(s.T, SELF_WARPS), c->fr_rblocks);
         LAUNCH(c, "route_select_screen", st,
-               route_select_fast(z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
-                                 c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 0, rblocks, st));
+               route_select_fast(z, z1, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx,
+                                 topk_gate, c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 0,
+                                 rblocks, st));
         if ((r = after_launch(c)) != MOP_OK) return r;
         LAUNCH(c, "route_select_resolve", st,
-               route_select_fast(z, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx, topk_gate,
-                                 c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 1, rblocks, st));
+               route_select_fast(z, nullptr, bias, static_cast<const bf16*>(x), c->fr_wrT, c->fr_xnorm, c->fr_wsq, topk_idx,
+                                 topk_gate, c->fr_todo, n_todo, stats, s.T, s.d, s.E, s.k, s.score_fn, s.bias_mode, 1,
+                                 rblocks, st));
         return after_launch(c);
     }
     LAUNCH(c, "route_score", st, route_score(static_cast<const bf16*>(x), W_r, z, s.T, s.d, s.E, c->sm_count, st));

@@ -451,7 +451,8 @@ __device__ __forceinline__ float key_error(float zz, float ez, int score_fn, int
 // zg: E floats (logits); clist: E ints, xs, ws: staging of the chains (RESOLVE only).
 template <bool RESOLVE, int Q>
 __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t* clist, float* xs, float* ws,
-                                            float* __restrict__ z, const float* __restrict__ bias,
+                                            float* __restrict__ z, const float* __restrict__ z1,
+                                            const float* __restrict__ bias,
                                             const bf16* __restrict__ x, const float* __restrict__ W_rT,
                                             const float* __restrict__ xnorm, float wmax, int32_t* __restrict__ idx,
                                             float* __restrict__ gate, int32_t* __restrict__ stats, int d, int E, int k,
@@ -465,6 +466,10 @@ __device__ __forceinline__ bool route_token(int t, int lane, float* zg, int32_t*
         kv[q] = 0.0f;
         if (e < E) {
             float zz = zrow[e];
+            if (z1) {                                // the logit GEMM left two partial sums over K: add, keep the sum
+                zz += z1[(size_t)t * E + e];
+                zrow[e] = zz;
+            }
             const float b = bias_mode ? bias[e] : 0.0f;
             if (bias_mode == 2) zz = __fadd_rn(zz, b);
             kv[q] = route_key_approx(zz, b, score_fn, bias_mode);
@@ -665,16 +670,16 @@ __device__ __forceinline__ float route_wmax(const float* __restrict__ wsq, int E
 constexpr int SCREEN_WARPS = 4;
 template <int Q>
 __global__ void __launch_bounds__(SCREEN_WARPS * 32) route_screen_kernel(
-    float* __restrict__ z, const float* __restrict__ bias, const float* __restrict__ xnorm,
-    const float* __restrict__ wsq, int32_t* __restrict__ idx, float* __restrict__ gate, int32_t* __restrict__ todo,
-    int32_t* __restrict__ n_todo, int T, int d, int E, int k, int score_fn, int bias_mode) {
+    float* __restrict__ z, const float* __restrict__ z1, const float* __restrict__ bias,
+    const float* __restrict__ xnorm, const float* __restrict__ wsq, int32_t* __restrict__ idx, float* __restrict__ gate,
+    int32_t* __restrict__ todo, int32_t* __restrict__ n_todo, int T, int d, int E, int k, int score_fn, int bias_mode) {
     extern __shared__ float sel_smem[];
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int t = blockIdx.x * SCREEN_WARPS + warp;
     if (t >= T) return;
     const float wmax = route_wmax(wsq, E, lane);
-    const bool done = route_token<false, Q>(t, lane, sel_smem + (size_t)warp * E, nullptr, nullptr, nullptr, z, bias, nullptr,
-                                            nullptr, xnorm, wmax, idx, gate, nullptr, d, E, k, score_fn, bias_mode);
+    const bool done = route_token<false, Q>(t, lane, sel_smem + (size_t)warp * E, nullptr, nullptr, nullptr, z, z1, bias,
+                                            nullptr, nullptr, xnorm, wmax, idx, gate, nullptr, d, E, k, score_fn, bias_mode);
     if (!done && lane == 0) todo[atomicAdd(n_todo, 1)] = t;
 }
 
@@ -695,21 +700,21 @@ __global__ void __launch_bounds__(SELF_WARPS * 32) route_resolve_kernel(
     float* ws = xs + SELF_XCHUNK;                           // the same chunk of up to SELF_CAND rows of W_r^T
     const float wmax = route_wmax(wsq, E, lane);
     for (int i = blockIdx.x * SELF_WARPS + warp; i < n; i += gridDim.x * SELF_WARPS) {
-        route_token<true, Q>(todo[i], lane, zg, clist, xs, ws, z, bias, x, W_rT, xnorm, wmax, idx, gate, stats, d, E, k,
-                             score_fn, bias_mode);
+        route_token<true, Q>(todo[i], lane, zg, clist, xs, ws, z, nullptr, bias, x, W_rT, xnorm, wmax, idx, gate, stats, d,
+                             E, k, score_fn, bias_mode);
         __syncwarp();
     }
 }
 
 // The two passes for the smallest supported Q >= ceil(E / 32).
 template <int Q>
-inline void route_select_fast_q(float* z, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
+inline void route_select_fast_q(float* z, const float* z1, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
                                 const float* wsq, int32_t* idx, float* gate, int32_t* todo, int32_t* n_todo,
                                 int32_t* stats, int T, int d, int E, int k, int score_fn, int bias_mode, int pass,
                                 int resolve_blocks, cudaStream_t st) {
     if (pass == 0) {
         route_screen_kernel<Q><<<ceil_div(T, SCREEN_WARPS), SCREEN_WARPS * 32, (size_t)SCREEN_WARPS * E * sizeof(float), st>>>(
-            z, bias, xnorm, wsq, idx, gate, todo, n_todo, T, d, E, k, score_fn, bias_mode);
+            z, z1, bias, xnorm, wsq, idx, gate, todo, n_todo, T, d, E, k, score_fn, bias_mode);
     } else {
         const size_t smem = (size_t)SELF_WARPS * (2 * E + SELF_SMEM_FLOATS) * sizeof(float);
         route_resolve_kernel<Q><<<resolve_blocks, SELF_WARPS * 32, smem, st>>>(z, bias, x, W_rT, xnorm, wsq, idx, gate, todo,
@@ -735,13 +740,13 @@ inline int route_resolve_resident(int E, int sm_count) {
     if (q <= 16) return route_resolve_resident_q<16>(E, sm_count);
     return route_resolve_resident_q<32>(E, sm_count);
 }
-inline void route_select_fast(float* z, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
+inline void route_select_fast(float* z, const float* z1, const float* bias, const bf16* x, const float* W_rT, const float* xnorm,
                               const float* wsq, int32_t* idx, float* gate, int32_t* todo, int32_t* n_todo, int32_t* stats,
                               int T, int d, int E, int k, int score_fn, int bias_mode, int pass, int resolve_blocks,
                               cudaStream_t st) {
     const int q = ceil_div(E, 32);
 #define MOP_ROUTE_Q(QQ)                                                                                                 \
-    route_select_fast_q<QQ>(z, bias, x, W_rT, xnorm, wsq, idx, gate, todo, n_todo, stats, T, d, E, k, score_fn, bias_mode, \
+    route_select_fast_q<QQ>(z, z1, bias, x, W_rT, xnorm, wsq, idx, gate, todo, n_todo, stats, T, d, E, k, score_fn, bias_mode, \
                             pass, resolve_blocks, st)
     if (q <= 2) MOP_ROUTE_Q(2);
     else if (q <= 4) MOP_ROUTE_Q(4);
