@@ -323,6 +323,16 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             if (t + n_clusters < total_tiles) nxt = decode(t + n_clusters);
             const int buf = it & 1;
             const uint32_t tphase = (uint32_t)(it >> 1) & 1u;
+            // F2: the gates of the tile's tokens (two dependent loads each) are fetched before the wait for the
+            // accumulator, so that their latency is hidden behind the main loop instead of paid per 32 tokens
+            float gpre[8];
+            if constexpr (KIND == TN_F2) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int tk = 32 * j + lane;
+                    gpre[j] = tk < ti.rows ? args.ep.gate[args.ep.row_src[ti.row0 + tk]] : 0.0f;
+                }
+            }
             bool ready = mbar_wait_warp(tfull_bar(buf), tphase, abort_flag, args.status, STATUS_WAIT_TMEM_FULL, lane);
             // the gate warp and its up warp meet at a named barrier below: they give up together or not at all
             if constexpr (KIND == TN_F1 || KIND == TN_F1G) ready = bar_vote_all(1 + (quarter & 1), 64, ready);
@@ -447,15 +457,14 @@ tn_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                 const int mcol = ti.mt * 256 + 128 * (int)rank + 32 * quarter;      // first output column of this warp
                 const bool m_ok = mcol < args.Mw;
                 uint16_t* st0 = reinterpret_cast<uint16_t*>(wbuf);
-#pragma unroll 1
-                for (int c = 0; c < ti.nmma; c += 32) {
+#pragma unroll
+                for (int j8 = 0; j8 < 8; ++j8) {
+                    const int c = 32 * j8;
+                    if (c >= ti.nmma) break;
                     tmem_ld32(taddr + c, v);
                     const int rows_left = ti.rows - c;
                     // gate of token (c + lane), handed round by shuffle
-                    float gmine = (KIND == TN_B4) ? 1.0f : 0.0f;
-                    if constexpr (KIND == TN_F2) {
-                        if (lane < rows_left) gmine = args.ep.gate[args.ep.row_src[ti.row0 + c + lane]];
-                    }
+                    const float gmine = (KIND == TN_F2) ? gpre[j8] : 1.0f;
 #pragma unroll
                     for (int tk = 0; tk < 32; ++tk) {
                         const float g = __shfl_sync(0xffffffffu, gmine, tk);
