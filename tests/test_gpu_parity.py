@@ -211,6 +211,25 @@ def test_an_overflowing_expert_does_not_reach_its_neighbours_gradients():
         assert torch.equal(clean.dX[~mine], bad.dX[~mine]) and torch.equal(clean.dgate[~mine], bad.dgate[~mine])
 
 
+@pytest.mark.parametrize("T,k,E", [(2048, 2, 24), (2049, 2, 24), (4096, 1, 1024), (1025, 4, 7), (4609, 1, 3)])
+def test_permutation_tables_on_both_sides_of_the_single_block_limit(T, k, E):
+    """Up to 8 units of 512 assignments the permutation runs in one block, beyond that in three kernels: the tables
+    must be the oracle's on both sides of that limit (and where the single block would not have the memory)."""
+    gen = torch.Generator().manual_seed(T + E)
+    idx = torch.stack([torch.randperm(E, generator=gen)[:k] for _ in range(T)]).to(torch.int32)
+    counts, offsets, perm_row, row_src = oracle.permute(idx.numpy(), E)
+    ctx = binding.Context(T, 64, E, k, 64)
+    dev = {n: torch.empty(s, dtype=torch.int32, device="cuda") for n, s in
+           (("counts", (E,)), ("offsets", (E + 1,)), ("perm_row", (T * k,)), ("row_src", (T * k,)))}
+    x = torch.randn((T, 64)).to(torch.bfloat16).cuda()
+    Xp = torch.empty((T * k, 64), dtype=torch.bfloat16, device="cuda")
+    binding.mop_moe_permute(ctx, x, idx.cuda(), dev["counts"], dev["offsets"], dev["perm_row"], dev["row_src"], Xp)
+    binding.mop_poll(ctx)
+    assert np.array_equal(dev["counts"].cpu().numpy(), counts) and np.array_equal(dev["offsets"].cpu().numpy(), offsets)
+    assert np.array_equal(dev["perm_row"].cpu().numpy(), perm_row) and np.array_equal(dev["row_src"].cpu().numpy(), row_src)
+    assert torch.equal(Xp.cpu(), x.cpu()[torch.from_numpy(row_src // k).long()])
+
+
 def test_zero_tokens_is_a_no_op():
     w = synth.small("c1_tiny", T=0, d=64, E=4, k=2, f=64, backward=True)
     host, inp, ctx, buf = run(w)
@@ -480,6 +499,8 @@ FAST_ROUTE = [
     synth.small("c3_trillion", T=300, d=192, E=1024, k=32, f=64, seed=63),                  # the selection's limits
     synth.small("c2_mid", T=257, d=64, E=64, k=32, f=64, seed=64),                          # half of the experts picked
     synth.small("c3_trillion", T=130, d=7168, E=384, k=8, f=64, seed=65),                   # the long chains of configs 3-5
+    synth.small("c3_trillion", T=600, d=448, E=64, k=4, f=64, seed=66),                     # one narrow tile of experts, K in halves
+    synth.small("c3_trillion", T=520, d=512, E=320, k=8, f=64, seed=67),                    # a wide tile and 64 more experts
 ]
 
 
