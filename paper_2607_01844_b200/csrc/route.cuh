@@ -298,14 +298,16 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) route_select_kernel(const floa
 //    This is a model, not a worst case (which is d u ||x|| ||w||): the realised maximum over millions
 //    of logits is 3 to 6.2 u ||x|| ||w|| on every shape tried, the tests assert it, and every logit that
 //    the kernel re-evaluates is compared with half the bound as it runs (mop_route_stats).
-//    In key space a logit error e moves sigmoid(z) + b by at most (s (1 - s) + e / 8) e + 4e-7.
-// 2. One warp per token selects the k largest approximate keys and gives every key the interval that
+//    In key space a logit error e moves sigmoid(z) + b by at most (s (1 - s) + e / 8) e + 4e-7; approximate
+//    keys are formed with the fast sigmoid, whose own error (below 1e-6) is added to that.
+// 2. Screening pass, one warp per token: the k largest approximate keys, every key with the interval that
 //    holds its exact value.  If the intervals of adjacent picks are disjoint and no other expert's
 //    interval reaches the weakest pick, the exact keys have the same order and the token is done
-//    (more than nine tenths of the tokens).  Otherwise the warp evaluates the contract's chain
-//    (__fmaf_rn, i ascending, W_r read through its transposed copy) for the experts in doubt, whose
-//    intervals become points, writes those logits over z~, and selects again, until nothing that
-//    matters overlaps.  Indices and their order are then those of the exact path.
+//    (more than nine tenths of the tokens).  The others are listed.  Resolving pass, one warp per listed
+//    token: it evaluates the contract's chain (__fmaf_rn, i ascending, W_r read through its transposed
+//    copy) for the experts in doubt, whose intervals become points and whose keys are the contract's,
+//    writes those logits over z~, and selects again, until nothing that matters overlaps.  Indices and
+//    their order are then those of the exact path.
 // 3. Gates are ratios of scores, not an order: a pick keeps its approximate logit unless that could move
 //    its gate by more than 5e-6 relative (score far from saturation), in which case its chain is
 //    evaluated too; the gates then agree with the exact path's to 1e-6 + 1e-5 g.
